@@ -1,0 +1,363 @@
+"""Pins for the CPU oracle: each test checks it against something other than itself —
+brute force, an identity of the paper, a closed form, exhaustive search, a hand-worked
+fixture, or a library routine."""
+
+import itertools
+import json
+import os
+
+import numpy as np
+import pytest
+
+from oracle import base_oracle as O
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def make_layer(seed, T=7, d=16, E=6, K=3, I=8, scale=1.0):
+    """Well-conditioned random layer (not the benchmark recipe: O(1) expert outputs)."""
+    r = np.random.default_rng(seed)
+    z = r.standard_normal((T, d))
+    logits = (r.standard_normal((T, E)) * 1.5).astype(np.float32)
+    Wg = r.standard_normal((E, I, d)) * scale / np.sqrt(d)
+    Wu = r.standard_normal((E, I, d)) * scale / np.sqrt(d)
+    Wd = r.standard_normal((E, d, I)) * scale / np.sqrt(I)
+    A = r.standard_normal((E, d)) * 0.7
+    b = r.standard_normal(E) * 0.3
+    ew = lambda u: (Wg[u], Wu[u], Wd[u])
+    return z, logits, A, b, ew
+
+
+# --------------------------------------------------------------------------- brute force: removal cost
+
+def test_removal_cost_is_with_minus_without_each_expert():
+    """Eq. individual_expert_damage: D_u equals the squared change of the layer output when expert u
+    alone is deleted (a single omission has no cross term)."""
+    z, logits, A, b, ew = make_layer(1)
+    E, K = logits.shape[1], 3
+    _, R, _, _, w = O.route_topk(logits, K)
+    a = O.contributions(z, R, w, ew)
+    D = O.true_removal_cost(a, R, E)
+    dense = O.dense_topk_moe(z, logits, ew, K)
+    for u in range(E):
+        without = O.layer_drop(z, logits, ew, K, {u})
+        brute = float(np.sum((dense - without) ** 2))
+        assert brute == pytest.approx(D[u], rel=1e-10, abs=1e-14)
+    assert D.sum() == pytest.approx(float(np.sum((a * a).sum(axis=2))), rel=1e-12)
+
+
+def test_layer_path_with_drop_rule_matches_independent_drop():
+    """The main path (forced active set, drop fill, paper gates) equals the separately written
+    'dense minus omitted contributions' layer, for every subset of omitted experts of size <= 2."""
+    z, logits, A, b, ew = make_layer(2)
+    E, K = logits.shape[1], 3
+    for om in list(itertools.combinations(range(E), 1)) + list(itertools.combinations(range(E), 2)):
+        mask = np.ones(E, np.uint8)
+        mask[list(om)] = 0
+        out = O.moe_decode_layer(z, logits, A, b, ew, K, E, fill=O.FILL_DROP, forced_mask=mask)
+        ref = O.layer_drop(z, logits, ew, K, set(om))
+        np.testing.assert_allclose(out["y"], ref, rtol=1e-12, atol=1e-14)
+
+
+# --------------------------------------------------------------------------- budget >= union reproduces dense
+
+@pytest.mark.parametrize("seed", [3, 4, 5])
+def test_budget_at_or_above_union_is_dense(seed):
+    r = np.random.default_rng(seed)
+    z, logits, A, b, ew = make_layer(seed, T=5, E=10, K=2)
+    logits[:, 6:] -= 8.0  # concentrate routing so that the union is smaller than E
+    K, E = 2, 10
+    _, R, _, _, _ = O.route_topk(logits, K)
+    union = sorted(set(R.ravel().tolist()))
+    assert len(union) < E
+    dense = O.dense_topk_moe(z, logits, ew, K)
+    for M in (len(union), len(union) + 1, E, E + 5):
+        out = O.moe_decode_layer(z, logits, A, b, ew, K, M)
+        np.testing.assert_allclose(out["y"], dense, rtol=1e-12, atol=1e-14)
+        assert out["n_dispatched"] == len(union)
+        assert out["dispatched"] == union
+        assert out["mask"].sum() == min(M, E)          # exactly M admitted
+        np.testing.assert_array_equal(np.sort(out["exec_ids"], axis=1), np.sort(R, axis=1))
+        np.testing.assert_allclose(out["exec_gates"].sum(axis=1), 1.0, rtol=1e-13)
+    # one below the union must change something
+    out = O.moe_decode_layer(z, logits, A, b, ew, K, len(union) - 1)
+    assert out["n_dispatched"] <= len(union) - 1
+    assert np.abs(out["y"] - dense).max() > 0
+
+
+# --------------------------------------------------------------------------- aggregation invariances
+
+def test_aggregation_is_permutation_invariant_over_the_batch():
+    z, logits, A, b, ew = make_layer(6, T=9)
+    K, M = 3, 3
+    base = O.moe_decode_layer(z, logits, A, b, ew, K, M)
+    perm = np.random.default_rng(0).permutation(z.shape[0])
+    out = O.moe_decode_layer(z[perm], logits[perm], A, b, ew, K, M)
+    np.testing.assert_allclose(out["scores"], base["scores"], rtol=1e-14)
+    assert set(out["selected"].tolist()) == set(base["selected"].tolist())
+    np.testing.assert_allclose(out["y"], base["y"][perm], rtol=1e-12, atol=1e-15)
+    np.testing.assert_allclose(out["costs"], base["costs"][perm], rtol=1e-14)
+
+
+def test_common_intercept_shift_keeps_selection():
+    z, logits, A, b, ew = make_layer(7)
+    s0 = O.moe_decode_layer(z, logits, A, b, ew, 3, 3)
+    s1 = O.moe_decode_layer(z, logits, A, b + 0.37, ew, 3, 3)
+    np.testing.assert_array_equal(s0["selected"], s1["selected"])
+    np.testing.assert_allclose(s1["scores"], s0["scores"] * np.exp(0.37), rtol=1e-12)
+
+
+# --------------------------------------------------------------------------- gates
+
+def test_gate_rules():
+    z, logits, A, b, ew = make_layer(8, T=12, E=8, K=3)
+    K, M = 3, 4
+    out = O.moe_decode_layer(z, logits, A, b, ew, K, M)
+    np.testing.assert_allclose(out["w"].sum(axis=1), 1.0, rtol=1e-14)
+    mask = out["mask"].astype(bool)
+    lost_any = False
+    for t in range(z.shape[0]):
+        Rt = out["R"][t].tolist()
+        ex = out["exec_ids"][t].tolist()
+        g = out["exec_gates"][t]
+        kept = [u for u in Rt if mask[u]]
+        assert len([u for u in ex if u >= 0]) == min(K, M)
+        assert all(mask[u] for u in ex if u >= 0)
+        assert set(kept) <= set(ex)
+        # router-rank order
+        lg = [logits[t, u] for u in ex if u >= 0]
+        assert lg == sorted(lg, reverse=True)
+        # kept routes keep their original weight exactly
+        for u in kept:
+            assert g[ex.index(u)] == pytest.approx(out["w"][t][Rt.index(u)], rel=1e-14)
+        if len(kept) == K:
+            assert g.sum() == pytest.approx(1.0, rel=1e-13)
+        else:
+            lost_any = True
+            assert g.sum() < 1.0     # each backfilled score is below the one it replaces
+    assert lost_any
+    ren = O.moe_decode_layer(z, logits, A, b, ew, K, M, gate_rule=O.GATE_RULE_RENORM)
+    np.testing.assert_allclose(ren["exec_gates"].sum(axis=1), 1.0, rtol=1e-13)
+    np.testing.assert_array_equal(ren["exec_ids"], out["exec_ids"])
+
+
+def test_budget_below_topk_leaves_empty_slots():
+    z, logits, A, b, ew = make_layer(9, E=8, K=3)
+    out = O.moe_decode_layer(z, logits, A, b, ew, 3, 2)
+    assert (out["exec_ids"][:, 2] == -1).all() and (out["exec_gates"][:, 2] == 0).all()
+    assert (out["exec_ids"][:, :2] >= 0).all()
+
+
+# --------------------------------------------------------------------------- selection = additive optimum
+
+def test_top_m_minimises_additive_error_by_exhaustive_search():
+    z, logits, A, b, ew = make_layer(10, T=6, E=8, K=2)
+    E, K, M = 8, 2, 3
+    _, R, _, _, w = O.route_topk(logits, K)
+    a = O.contributions(z, R, w, ew)
+    D = O.true_removal_cost(a, R, E)
+    best = min(itertools.combinations(range(E), M), key=lambda S: sum(D[u] for u in range(E) if u not in S))
+    ids, mask = O.select_top(D, M)
+    assert set(ids.tolist()) == set(best)
+    assert list(D[ids]) == sorted(D[ids], reverse=True)
+    # exact error of Eq. error_decomposition == squared output change of deleting the omitted set
+    dense = O.dense_topk_moe(z, logits, ew, K)
+    for S in itertools.combinations(range(E), M):
+        m = np.zeros(E, np.uint8)
+        m[list(S)] = 1
+        tot, indiv, cross = O.exact_error(a, R, m)
+        om = set(range(E)) - set(S)
+        brute = float(np.sum((dense - O.layer_drop(z, logits, ew, K, om)) ** 2))
+        assert tot == pytest.approx(brute, rel=1e-10)
+        assert tot == pytest.approx(indiv + cross, rel=1e-10, abs=1e-14)
+        # individual damage restricted to omitted experts that were routed
+        assert indiv == pytest.approx(sum(D[u] for u in om), rel=1e-10)
+
+
+def test_select_ties_and_clipping():
+    ids, mask = O.select_top(np.array([1.0, 3.0, 3.0, 0.0, 0.0]), 4)
+    assert ids.tolist() == [1, 2, 0, 3] and mask.tolist() == [1, 1, 1, 1, 0]
+    ids, mask = O.select_top(np.array([1.0, 2.0]), 9)
+    assert ids.tolist() == [1, 0] and mask.sum() == 2
+    ids, _ = O.select_top(np.array([1.0, np.nan, 2.0]), 2)
+    assert ids.tolist() == [2, 0]
+
+
+def test_cross_term_identity():
+    """rho - 1 = c-bar (|U|_eff - 1), 1 <= |U|_eff <= |U|, rho = 1 for a single omission."""
+    r = np.random.default_rng(11)
+    for n in (1, 2, 3, 6):
+        a = r.standard_normal((n, 12)) * r.uniform(0.1, 3.0, size=(n, 1))
+        rho, cbar, eff = O.cross_term_stats(a)
+        assert rho - 1 == pytest.approx(cbar * (eff - 1), abs=1e-12)
+        assert 1 - 1e-12 <= eff <= n + 1e-12
+        if n == 1:
+            assert rho == pytest.approx(1.0)
+    same = np.tile(r.standard_normal(12), (4, 1))[:, :] * 1.0
+    assert O.cross_term_stats(same)[2] == pytest.approx(4.0)
+
+
+def test_energy_retained_bounds():
+    r = np.random.default_rng(12)
+    D = r.uniform(size=10)
+    _, best = O.select_top(D, 4)
+    assert O.energy_retained(best, D, 4) == pytest.approx(1.0)
+    for _ in range(20):
+        m = np.zeros(10, np.uint8)
+        m[r.choice(10, 4, replace=False)] = 1
+        assert 0.0 <= O.energy_retained(m, D, 4) <= 1.0 + 1e-15
+
+
+# --------------------------------------------------------------------------- predictor closed forms
+
+def test_zero_predictor_gives_squared_router_weight_score():
+    z, logits, A, b, ew = make_layer(13, T=10)
+    K, E = 3, logits.shape[1]
+    _, R, _, _, w = O.route_topk(logits, K)
+    costs = O.predict_costs(z, R, w, np.zeros_like(A), np.zeros_like(b))
+    ref = np.zeros(E)
+    np.add.at(ref, R.ravel(), (w ** 2).ravel())
+    np.testing.assert_allclose(O.aggregate(costs), ref, rtol=1e-14)
+    # static energy: a = 0, b = log mu
+    mu = np.random.default_rng(0).uniform(0.5, 2.0, E)
+    costs = O.predict_costs(z, R, w, np.zeros_like(A), np.log(mu))
+    np.testing.assert_allclose(O.aggregate(costs), ref * mu, rtol=1e-13)
+    assert (costs[np.arange(10)[:, None], R] > 0).all()
+    off = np.ones_like(costs, bool)
+    off[np.arange(10)[:, None], R] = False
+    assert (costs[off] == 0).all()
+
+
+def test_one_hot_predictor_reads_one_coordinate_of_normalised_input():
+    z, logits, A, b, ew = make_layer(14)
+    K, E, d = 3, logits.shape[1], z.shape[1]
+    _, R, _, _, w = O.route_topk(logits, K)
+    A1 = np.zeros((E, d))
+    for u in range(E):
+        A1[u, (3 * u + 1) % d] = 2.0
+    costs = O.predict_costs(z, R, w, A1, b)
+    for t in range(z.shape[0]):
+        zn = z[t] / np.linalg.norm(z[t])
+        for k in range(K):
+            u = R[t, k]
+            assert costs[t, u] == pytest.approx(w[t, k] ** 2 * np.exp(2.0 * zn[(3 * u + 1) % d] + b[u]), rel=1e-13)
+    # scaling the token leaves the cost unchanged (input is normalised)
+    costs2 = O.predict_costs(z * 7.5, R, w, A1, b)
+    np.testing.assert_allclose(costs2, costs, rtol=1e-12)
+
+
+def test_fig2_style_constructed_example():
+    with open(os.path.join(GOLDEN, "fig2_constructed.json")) as f:
+        g = json.load(f)
+    E, K, M = g["experts"], g["K"], g["M"]
+    routes, weights = np.array(g["routes"]), np.array(g["weights"])
+    T = routes.shape[0]
+    logits = np.full((T, E), -30.0, np.float32)
+    for t in range(T):
+        logits[t, routes[t, 0]] = np.float32(np.log(weights[t, 0] / weights[t, 1]))
+        logits[t, routes[t, 1]] = 0.0
+    d = 4
+    z = np.ones((T, d))
+    ew = lambda u: (np.eye(d) * (u + 1), np.eye(d), np.eye(d))
+    out = O.moe_decode_layer(z, logits, np.zeros((E, d)), np.log(np.array(g["predicted_energy"])), ew, K, M)
+    np.testing.assert_array_equal(out["R"], routes)
+    np.testing.assert_allclose(out["w"], weights, rtol=1e-6)
+    assert sorted(set(out["R"][:, 0].tolist())) == g["top1_union"]
+    np.testing.assert_allclose(out["scores"], g["scores"], rtol=1e-6, atol=1e-12)
+    assert out["selected"].tolist() == g["selected_desc"]
+    assert 2 not in out["R"][:, 0]               # e3 is never a top-1 expert, yet selected
+    # token 3 loses e5 (id 4): keeps e3 (id 2) and backfills with its next-preferred active expert
+    assert out["exec_ids"][3].tolist() == [2, 0]
+    assert out["exec_gates"][3][0] == pytest.approx(0.45, rel=1e-6)
+    assert out["exec_gates"][3].sum() < 0.46
+
+
+# --------------------------------------------------------------------------- expert function
+
+def test_swiglu_closed_form_orientation():
+    """d=2, I=1: E(z) = W_down * silu(g z0) * (u z1): catches a transposed operand or swapped gate/up."""
+    g_, u_ = 1.7, -0.6
+    Wg, Wu, Wd = np.array([[g_, 0.0]]), np.array([[0.0, u_]]), np.array([[2.0], [-3.0]])
+    z = np.array([[0.9, 1.3]])
+    s = g_ * 0.9
+    h = s / (1 + np.exp(-s)) * (u_ * 1.3)
+    np.testing.assert_allclose(O.expert_ffn(z, Wg, Wu, Wd), [[2.0 * h, -3.0 * h]], rtol=1e-14)
+
+
+def test_primitives_against_torch():
+    torch = pytest.importorskip("torch")
+    import torch.nn.functional as F
+    r = np.random.default_rng(15)
+    x = r.standard_normal((5, 12))
+    Wg, Wu, Wd = r.standard_normal((7, 12)), r.standard_normal((7, 12)), r.standard_normal((12, 7))
+    tx, tg, tu, td = (torch.from_numpy(a) for a in (x, Wg, Wu, Wd))
+    ref = (F.silu(tx @ tg.T) * (tx @ tu.T)) @ td.T
+    np.testing.assert_allclose(O.expert_ffn(x, Wg, Wu, Wd), ref.numpy(), rtol=1e-12)
+    logits = r.standard_normal((6, 9)).astype(np.float32)
+    order, R, q, S, w = O.route_topk(logits, 3)
+    tv, ti = torch.topk(torch.softmax(torch.from_numpy(logits).double(), dim=1), 3, dim=1)
+    np.testing.assert_array_equal(R, ti.numpy())
+    np.testing.assert_allclose(w, (tv / tv.sum(dim=1, keepdim=True)).numpy(), rtol=1e-12)
+    np.testing.assert_array_equal(order, torch.argsort(torch.from_numpy(logits), dim=1, descending=True, stable=True).numpy())
+    zz = r.standard_normal((4, 12))
+    np.testing.assert_allclose(O.normalise(zz), F.normalize(torch.from_numpy(zz), dim=1).numpy(), rtol=1e-14)
+    np.testing.assert_allclose(O.router_logits(x, Wg, np.arange(7.0)),
+                               (tx @ tg.T + torch.arange(7.0)).float().numpy(), rtol=1e-6)
+    h = r.standard_normal((4, 12))
+    np.testing.assert_allclose(O.stack_next_hidden(zz, h), F.rms_norm(torch.from_numpy(zz + h), (12,), eps=0).numpy(),
+                               rtol=1e-12)
+
+
+# --------------------------------------------------------------------------- calibration
+
+def test_ridge_matches_least_squares_and_recovers_planted_model():
+    r = np.random.default_rng(16)
+    n, d = 400, 10
+    X = r.standard_normal((n, d))
+    X /= np.linalg.norm(X, axis=1, keepdims=True)
+    a_true, b_true = r.standard_normal(d), 0.8
+    y = X @ a_true + b_true
+    a, b = O.ridge_fit(X, y, 1e-12)
+    np.testing.assert_allclose(a, a_true, rtol=1e-6, atol=1e-8)
+    assert b == pytest.approx(b_true, rel=1e-6)
+    yn = y + 0.1 * r.standard_normal(n)
+    a, b = O.ridge_fit(X, yn, 1e-10)
+    sol = np.linalg.lstsq(np.hstack([X, np.ones((n, 1))]), yn, rcond=None)[0]
+    np.testing.assert_allclose(np.append(a, b), sol, rtol=1e-6, atol=1e-8)
+    # shrinkage: the coefficient norm decreases with lambda
+    norms = [np.linalg.norm(O.ridge_fit(X, yn, lam)[0]) for lam in (1e-4, 1e-2, 1.0, 100.0)]
+    assert norms == sorted(norms, reverse=True)
+
+
+def test_fit_predictor_against_brute_force_removal_costs():
+    """Fit on routed calibration pairs; exp(s-hat) is unbiased on them and beats the static score
+    out of sample when the energy depends on the token's direction."""
+    r = np.random.default_rng(17)
+    d, E, K, I, n = 12, 4, 2, 6, 1500
+    Wg = r.standard_normal((E, I, d)) / np.sqrt(d)
+    v = r.standard_normal((E, d))
+    v /= np.linalg.norm(v, axis=1, keepdims=True)
+    Wg = Wg + 1.5 * v[:, None, :]                 # planted direction: energy depends on z . v_u
+    Wu = r.standard_normal((E, I, d)) / np.sqrt(d)
+    Wd = r.standard_normal((E, d, I)) / np.sqrt(I)
+    ew = lambda u: (Wg[u], Wu[u], Wd[u])
+    z = r.standard_normal((n, d))
+    logits = r.standard_normal((n, E)).astype(np.float32)
+    A, b = O.fit_predictor(z[:1000], logits[:1000], ew, K, E, lam=1e-2)
+    zt, lt = z[1000:], logits[1000:]
+    _, R, _, _, w = O.route_topk(lt, K)
+    a = O.contributions(zt, R, w, ew)
+    true_c = (a * a).sum(axis=2)                   # brute-force per-pair removal cost
+    pred_c = np.take_along_axis(O.predict_costs(zt, R, w, A, b), R, axis=1)
+    mu = np.array([np.mean([(O.expert_ffn(z[i:i + 1], *ew(u)) ** 2).sum() for i in range(200)]) for u in range(E)])
+    static_c = w ** 2 * mu[R]
+    err_pred = np.mean((np.log(pred_c) - np.log(true_c)) ** 2)
+    err_static = np.mean((np.log(static_c) - np.log(true_c)) ** 2)
+    assert err_pred < 0.8 * err_static
+    # unbiased in the mean on the calibration pairs
+    _, Rc, _, _, wc = O.route_topk(logits[:1000], K)
+    ac = O.contributions(z[:1000], Rc, wc, ew)
+    tc = (ac * ac).sum(axis=2) / wc ** 2
+    pc = np.take_along_axis(O.predict_costs(z[:1000], Rc, wc, A, b), Rc, axis=1) / wc ** 2
+    for u in range(E):
+        assert pc[Rc == u].mean() == pytest.approx(tc[Rc == u].mean(), rel=1e-9)
