@@ -1,0 +1,411 @@
+#!/usr/bin/env python
+"""Benchmark of the BASE batched MoE decode layer on B200.
+
+One "step" is one pass of the whole hot path (router + predictor GEMV, routing kernel, gather,
+grouped SwiGLU FFN over the dispatched experts, combine) over one decode batch of synthetic
+input. Default workload: the Qwen3-30B-A3B-shaped layer, batch 64, expert budget 32.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--workload qwen3|mid|mixtral|tiny|qwen3_stack] [--budget M] [--batch T] [--sweep]
+
+Prints ONE JSON line (rank 0). Timing: CUDA events on the launching stream around K graph
+replays; L2 is kept cold by rotating independently seeded weight replicas whose dispatched
+bytes exceed the L2 size several times over.
+"""
+
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            with open(p) as f:
+                return json.load(f), "measured"
+        except Exception:
+            pass
+    return {"hbm_gbs": FALLBACK_HBM_GBS, "bf16_tflops": 1590.0}, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clock/throttle sampler running during the timed region (read-only queries)."""
+
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.path = None
+
+    def __enter__(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.gpu)], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+        return self
+
+    def __exit__(self, *exc):
+        if self.proc is not None:
+            time.sleep(0.15)
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
+
+    def summary(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if not self.path or not os.path.exists(self.path):
+            return out
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in open(self.path):
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                sm.append(float(parts[1]))
+                mx.append(float(parts[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        try:
+            os.unlink(self.path)
+        except OSError:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+def algorithmic_bytes(cfg, T, n_dispatched, out_bytes=2):
+    """Bytes the method must move for one step: dispatched experts' weights, router and predictor rows,
+    hidden states in, layer output out."""
+    return (n_dispatched * cfg.expert_bytes + 2 * cfg.E * cfg.d * 2 + T * cfg.d * 2 + T * cfg.d * out_bytes)
+
+
+def ffn_algorithmic_bytes(cfg, T, n_dispatched):
+    """Bytes of the FFN kernels alone: weights of the dispatched experts + activations in + result out."""
+    return n_dispatched * cfg.expert_bytes + T * cfg.d * 2 + T * cfg.d * 4
+
+
+# ------------------------------------------------------------------------------------------ oracle arm
+
+def oracle_step_seconds(cfg, T, M, repeats, layer=0):
+    """Time the CPU oracle, as it stands, on one full step of the workload. Returns (best seconds, cores)."""
+    from oracle import base_oracle as O
+    from paper_2609_36222_b200 import workloads as wl
+
+    hid = wl.hidden_bits(cfg, T, layer=layer)
+    small = wl.small_tensors(cfg, layer=layer)
+    z = wl.bf16_bits_to_f64(hid)
+    rw, A = wl.bf16_bits_to_f64(small["router_w"]), wl.bf16_bits_to_f64(small["pred_A"])
+    rb, pb = small["router_bias"].astype(np.float64), small["pred_b"].astype(np.float64)
+    cache = {}
+
+    def ew(u):
+        if u not in cache:
+            bits = wl.expert_weights_host(cfg, u, layer=layer)
+            cache[u] = {k: wl.bf16_bits_to_f32(v) for k, v in bits.items()}   # storage-precision values
+        c = cache[u]
+        return c["w_gate"], c["w_up"], c["w_down"]
+
+    # materialise the inputs (not timed: they are the workload, not the method)
+    logits0 = O.router_logits(z, rw, rb)
+    res = O.moe_decode_layer(z, logits0, A, pb, ew, cfg.K, M)
+    times = []
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        logits = O.router_logits(z, rw, rb)
+        res = O.moe_decode_layer(z, logits, A, pb, ew, cfg.K, M)
+        times.append(time.perf_counter() - t0)
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+    except Exception:
+        cores = os.cpu_count() or 1
+    return min(times), cores, res["n_dispatched"]
+
+
+def run_reference(args, cfg, T, M):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    reps = max(1, min(args.steps, 3))
+    best, cores, nd = oracle_step_seconds(cfg, T, M, reps)
+    us = best * 1e6
+    line = {
+        "impl": "reference", "metric": "moe_decode_layer_us_per_step", "value": us, "unit": "us/step",
+        "n_gpus": args.gpus, "steps": reps, "warmup": 1, "ms_per_step": us / 1e3, "higher_is_better": False,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{cfg.name} layer d={cfg.d} E={cfg.E} K={cfg.K} I={cfg.I} batch={T} budget={M}",
+                   "n_dispatched": nd},
+        "cpu_baseline": {"value": us, "unit": "us/step", "cores": cores, "kind": "oracle",
+                         "sample": f"{reps} full step(s) of the workload (replica 0), best of {reps}"},
+        "e2e": {"value": us, "unit": "us/step", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------ CUDA arm
+
+def run_ours(args, cfg, T, M):
+    import torch
+
+    import __graft_entry__ as entry
+    entry.build()
+    from paper_2609_36222_b200 import binding as B
+    from paper_2609_36222_b200 import workloads as wl
+    from paper_2609_36222_b200.layer import DeviceLayer, bits_to_device
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the CUDA path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    peaks, peak_kind = measured_peaks()
+    hbm_peak = float(peaks.get("hbm_gbs", FALLBACK_HBM_GBS))
+
+    stack = cfg.layers > 1
+    # Replicas: independent seeded layers rotated between steps so no step finds its weights in L2.
+    if stack:
+        n_rep = cfg.layers
+    else:
+        n_rep = max(2, min(8, int(np.ceil(4 * 126e6 / max(1, min(M, cfg.E) * cfg.expert_bytes))) + 1))
+        if cfg.E * cfg.expert_bytes * n_rep > 40e9:
+            n_rep = max(2, int(40e9 // (cfg.E * cfg.expert_bytes)))
+    shape = (cfg.d, cfg.E, cfg.K, cfg.I)
+    ws = B.alloc_workspace(max(B.layer_workspace_bytes(*shape, T), B.stack_workspace_bytes(*shape, T)), dev)
+    base_layer = rank * 1000
+    layers = [DeviceLayer(cfg, dev, layer=base_layer + r, T_max=T, workspace=ws) for r in range(n_rep)]
+    hidden = [bits_to_device(wl.hidden_bits(cfg, T, layer=base_layer + r), dev) for r in range(n_rep)]
+    out = torch.empty(T, cfg.d, dtype=torch.bfloat16, device=dev)
+    nd_buf = torch.zeros(max(n_rep, 1), dtype=torch.int32, device=dev)
+    stream = torch.cuda.Stream(device=dev)
+
+    dbgs = []
+    for r in range(n_rep):
+        dbg = B.LayerDebug()
+        dbg.n_dispatched = nd_buf[r:].data_ptr()
+        dbgs.append(dbg)
+
+    def step_eager(i, budget=M):
+        if stack:
+            B.base_moe_decode_stack(shape, [l.weights for l in layers], hidden[0], budget, out, ws,
+                                    n_dispatched=nd_buf, stream=stream)
+        else:
+            r = i % n_rep
+            B.base_moe_decode_layer(shape, layers[r].weights, hidden[r], budget, out, ws, debug=dbgs[r], stream=stream)
+
+    # one eager pass (also fills n_dispatched per replica), then capture one graph per replica
+    with torch.cuda.stream(stream):
+        for r in range(1 if stack else n_rep):
+            step_eager(r)
+    stream.synchronize()
+    launches_per_step = B.last_launch_count()
+    nd = nd_buf.cpu().numpy().astype(np.int64)
+    mean_nd = float(nd.mean())
+
+    def capture(budget):
+        graphs = []
+        for r in range(1 if stack else n_rep):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                step_eager(r, budget)
+            graphs.append(g)
+        return graphs
+
+    def timed(graphs, steps, warmup):
+        with torch.cuda.stream(stream):
+            for i in range(warmup):
+                graphs[i % len(graphs)].replay()
+            stream.synchronize()
+            if dist is not None:
+                dist.barrier()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for i in range(steps):
+                graphs[(warmup + i) % len(graphs)].replay()
+            e1.record(stream)
+            e1.synchronize()
+            torch.cuda.synchronize()
+            if dist is not None:
+                dist.barrier()
+        return e0.elapsed_time(e1) / steps   # ms per step
+
+    graphs = capture(M)
+    with ClockSampler(local) as clocks:
+        ms = timed(graphs, args.steps, args.warmup)
+        # keep the sampler alive long enough to see the load when the run is very short
+        if ms * args.steps < 300:
+            timed(graphs, max(args.steps, int(300 / max(ms, 1e-3))), 0)
+    clk = clocks.summary()
+    if dist is not None:
+        t = torch.tensor([ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+
+    # ---- per-kernel pass for the roofline: the library records the caller's events around the FFN kernels
+    n_prof = min(args.steps, 40)
+    ffn_us = None
+    if hasattr(B.lib(), "base_profile_ffn_events"):
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_prof)]
+        with torch.cuda.stream(stream):
+            for i in range(3):
+                step_eager(i)
+            for i, (a, b) in enumerate(evs):
+                a.record(stream)   # create both handles before the library records them again
+                b.record(stream)
+                B.lib().base_profile_ffn_events(a.cuda_event, b.cuda_event)
+                step_eager(3 + i)
+            B.lib().base_profile_ffn_events(None, None)
+        stream.synchronize()
+        # (in a stack every layer re-records the pair, so this is the last layer's FFN)
+        ffn_us = statistics.mean(a.elapsed_time(b) for a, b in evs) * 1e3
+
+    # ---- unlimited budget (dense batch-union step) for the speed-up, same protocol
+    ms_dense = None
+    if not args.no_dense:
+        with torch.cuda.stream(stream):
+            for r in range(1 if stack else n_rep):
+                step_eager(r, cfg.E)
+        stream.synchronize()
+        nd_dense = float(nd_buf.cpu().numpy().astype(np.int64).mean())
+        ms_dense = timed(capture(cfg.E), args.steps, args.warmup)
+
+    # ---- end to end through the host entry point (pinned host buffers, copies inside the timed region)
+    e2e = None
+    if not stack:
+        hws = B.alloc_workspace(B.layer_host_workspace_bytes(*shape, T), dev)
+        h_in = [torch.from_numpy(wl.hidden_bits(cfg, T, layer=base_layer + r).view(np.int16)).view(torch.bfloat16).pin_memory()
+                for r in range(n_rep)]
+        h_out = torch.empty(T, cfg.d, dtype=torch.bfloat16).pin_memory()
+        h_nd = torch.zeros(1, dtype=torch.int32).pin_memory()
+        for i in range(args.warmup):
+            B.base_moe_decode_layer_host(shape, layers[i % n_rep].weights, h_in[i % n_rep], M, h_out, hws,
+                                         h_n_dispatched=h_nd, stream=stream)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for i in range(args.steps):
+            r = (args.warmup + i) % n_rep
+            B.base_moe_decode_layer_host(shape, layers[r].weights, h_in[r], M, h_out, hws, h_n_dispatched=h_nd,
+                                         stream=stream)
+        e2e_us = (time.perf_counter() - t0) / args.steps * 1e6
+        if dist is not None:
+            t = torch.tensor([e2e_us], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_us = float(t.item())
+        e2e = {"value": e2e_us / world, "unit": "us/step", "h2d_bytes_per_step": T * cfg.d * 2,
+               "d2h_bytes_per_step": T * cfg.d * 2 + 4}
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    us = ms * 1e3
+    per_layer_us = us / (cfg.layers if stack else 1)
+    step_bytes = algorithmic_bytes(cfg, T, mean_nd)
+    gbs = step_bytes / (per_layer_us * 1e-6) / 1e9
+    line = {
+        "metric": "moe_decode_layer_us_per_step", "value": us / world, "unit": "us/step", "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": False,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {
+            "workload": f"{cfg.name} {'stack L=%d ' % cfg.layers if stack else 'layer '}d={cfg.d} E={cfg.E} K={cfg.K} "
+                        f"I={cfg.I} batch={T} budget={M}",
+            "l2": f"cold: {n_rep} independently seeded weight replicas rotated between steps "
+                  f"({mean_nd * cfg.expert_bytes / 1e6:.0f} MB dispatched per step vs 126 MB L2)",
+            "n_dispatched_mean": mean_nd, "replicas": n_rep, "timing": "CUDA events around graph replays",
+            "multi_gpu": "independent replicas per rank, no collective" if world > 1 else "single GPU",
+        },
+        "hbm": {"algorithmic_bytes_per_step": step_bytes, "gbs": gbs, "frac_of_nominal_8tbs": gbs / NOMINAL_HBM_GBS,
+                "frac_of_measured_copy": gbs / hbm_peak, "peak_kind": peak_kind},
+        "clocks": {"sm_mhz": clk["sm_mhz"], "sm_max_mhz": clk["sm_max_mhz"], "reasons": clk["reasons"]},
+        "gpu_launches": launches_per_step * args.steps,
+    }
+    if ms_dense is not None:
+        line["unlimited_budget"] = {"us_per_step": ms_dense * 1e3, "n_dispatched_mean": nd_dense,
+                                    "speedup_from_budget": ms_dense / ms}
+    if e2e is not None:
+        line["e2e"] = e2e
+    if ffn_us is not None:
+        fb = ffn_algorithmic_bytes(cfg, T, mean_nd)
+        ach = fb / (ffn_us * 1e-6) / 1e9
+        line["roofline"] = {"bound": "hbm", "kernel": "grouped SwiGLU FFN (gate/up + down)", "achieved": ach,
+                            "peak": hbm_peak, "unit": "GB/s", "frac": ach / hbm_peak, "traffic": None,
+                            "us_per_launch": ffn_us, "peak_kind": f"of {peak_kind}",
+                            "algorithmic_bytes_per_launch": fb}
+    # CPU baseline: the oracle, as it stands, on this machine's host cores
+    if not args.no_cpu:
+        reps = 2 if cfg.expert_bytes < (64 << 20) else 1
+        best, cores, _ = oracle_step_seconds(cfg if not stack else wl.CONFIGS["qwen3"], T, M, reps)
+        scale = cfg.layers if stack else 1
+        line["cpu_baseline"] = {"value": best * 1e6 * scale, "unit": "us/step", "cores": cores, "kind": "oracle",
+                                "sample": f"{reps} full layer step(s), best of {reps}" +
+                                          (f", x{scale} layers extrapolated" if stack else "")}
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="qwen3")
+    ap.add_argument("--budget", type=int, default=32)
+    ap.add_argument("--batch", type=int, default=None)
+    ap.add_argument("--no-cpu", action="store_true", help="skip the oracle timing")
+    ap.add_argument("--no-dense", action="store_true", help="skip the unlimited-budget run")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    from paper_2609_36222_b200 import workloads as wl
+    cfg = wl.CONFIGS[args.workload]
+    T = args.batch or cfg.T
+    M = args.budget
+    if args.impl == "reference":
+        run_reference(args, cfg, T, M)
+    else:
+        run_ours(args, cfg, T, M)
+
+
+if __name__ == "__main__":
+    main()

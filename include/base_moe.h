@@ -1,0 +1,197 @@
+/*
+ * base_moe.h -- C ABI of the B200 (sm_100a) batched MoE decode layer with batch-aware expert
+ * selection by predicted removal error (BASE).
+ *
+ * One decode step of one MoE layer, for a batch of T tokens (one per active sequence):
+ *   route      top-K router over N experts, weights = softmax scores renormalised over the top-K
+ *              (problem formulation, Sec. 3.1)
+ *   predict    c[t,u] = w[t,u]^2 * exp(a_u . z_t/||z_t|| + b_u) for the routed pairs
+ *              (Eq. log_energy_predictor, Sec. 3.4; kernel description in App. "Custom GPU Kernels")
+ *   aggregate  D[u] = sum_t c[t,u]                                  (same equation)
+ *   select     active set A = the M experts with the largest D[u]   (Sec. 3.4 / 3.5)
+ *   restrict   every token executes its K highest-ranked experts inside A; the gate of an executed
+ *              expert is its own router score over the denominator of the token's ORIGINAL top-K
+ *              (inference procedure, Sec. 3.5)
+ *   execute    y_t = sum_{u in R'_t} g[t,u] * W_down,u( silu(W_gate,u z_t) * (W_up,u z_t) ), reading
+ *              only the weights of experts that received a token (latency model, Eq. moe_latency)
+ *
+ * Conventions for every entry point
+ *   - Pointers are DEVICE pointers unless the name starts with h_. The caller owns every buffer.
+ *     Unless stated otherwise the library allocates no device memory and never synchronises: work
+ *     is enqueued on `stream` (a cudaStream_t passed as void*; NULL = the legacy default stream).
+ *   - "bf16" buffers hold IEEE bfloat16 bit patterns, row-major, innermost dimension contiguous.
+ *   - Every tensor base address must be 16-byte aligned; d and I must be multiples of 64.
+ *   - Return value: BASE_OK or an error code below. Nothing is enqueued when an argument check
+ *     fails. The library never aborts and never throws. Conditions only the device can see
+ *     (a non-finite score, a bounded wait that ran out) are OR-ed into the optional int32 status
+ *     word of base_layer_debug as BASE_DEV_* bits.
+ */
+#ifndef BASE_MOE_H
+#define BASE_MOE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+  BASE_OK = 0,
+  BASE_ERR_INVALID_ARG = 1,        /* null / misaligned pointer, non-positive size, bad enum */
+  BASE_ERR_UNSUPPORTED = 2,        /* shape outside the compiled limits (see each call) */
+  BASE_ERR_WORKSPACE_TOO_SMALL = 3,
+  BASE_ERR_CUDA = 4                /* a CUDA call failed; base_last_cuda_error() has the code */
+};
+
+enum {                             /* bits of the device status word */
+  BASE_DEV_NONFINITE_SCORE = 1,    /* some aggregated score was NaN/Inf (NaN ranks last) */
+  BASE_DEV_WAIT_EXPIRED = 2,       /* a bounded wait inside a kernel gave up; output is invalid */
+  BASE_DEV_BAD_INDEX = 4           /* an expert id outside [0,E) was met and skipped */
+};
+
+enum { BASE_GATE_PAPER = 0,        /* Sec. 3.5: original top-K denominator (gates may sum to < 1) */
+       BASE_GATE_RENORM = 1 };     /* renormalise over the executed experts (OEA-style variant) */
+enum { BASE_FILL_BACKFILL = 0,     /* Sec. 3.5: next-preferred experts inside the active set */
+       BASE_FILL_DROP = 1 };       /* fill-rule ablation: unavailable routes are removed */
+
+/*
+ * Predicted removal costs of the routed pairs (Eq. log_energy_predictor; scoring kernel of
+ * App. "Custom GPU Kernels").
+ *   hidden_bf16 [T,d] bf16   token inputs z_t (normalised inside the kernel, once per token)
+ *   topk_ids    [T,K] int32  routed experts R_t; an id outside [0,E) is skipped
+ *   topk_w      [T,K] fp32   router weights w[t,u], normalised over R_t
+ *   pred_A_bf16 [E,d] bf16, pred_b [E] fp32   predictor rows a_u and intercepts b_u
+ *   costs       [T,E] fp32   OUT: c[t,u] for u in R_t, exactly 0 elsewhere
+ * Limits: d % 8 == 0, K <= 64. One CTA per token, one warp per routed expert, 128-bit loads.
+ */
+int base_predict_costs(const void* hidden_bf16, const int32_t* topk_ids, const float* topk_w,
+                       const void* pred_A_bf16, const float* pred_b, float* costs,
+                       int T, int d, int E, int K, void* stream);
+
+/*
+ * Batch aggregation and top-M selection (Eq. log_energy_predictor; Sec. 3.5; selection kernel of
+ * App. "Custom GPU Kernels"). One CTA, no host round trip.
+ *   costs        [T,E] fp32
+ *   budget       M >= 1; values above E are clipped to E; exactly min(M,E) experts are admitted
+ *   scores       [E] fp32   OUT: D[u] = sum_t costs[t,u]
+ *   selected_ids [min(M,E)] int32  OUT: admitted experts by descending score, equal scores by
+ *                ascending id, NaN scores last
+ *   active_mask  [E] uint8  OUT: 1 for admitted experts
+ * Limits: E <= 1024.
+ */
+int base_aggregate_select(const float* costs, int T, int E, int budget, float* scores,
+                          int32_t* selected_ids, uint8_t* active_mask, void* stream);
+
+typedef struct {
+  int d;   /* model width */
+  int E;   /* routed experts (the paper's N) */
+  int K;   /* router top-K */
+  int I;   /* SwiGLU intermediate width of one expert */
+} base_layer_shape;
+
+typedef struct {
+  const void* router_w;     /* [E,d] bf16; may be NULL when router_logits are supplied */
+  const float* router_bias; /* [E] fp32 or NULL (= 0) */
+  const void* pred_A;       /* [E,d] bf16 */
+  const float* pred_b;      /* [E] fp32 */
+  const void* w_gate;       /* [E,I,d] bf16 */
+  const void* w_up;         /* [E,I,d] bf16 */
+  const void* w_down;       /* [E,d,I] bf16 */
+} base_layer_weights;
+
+/* Optional copies of the intermediates (any member may be NULL). */
+typedef struct {
+  float* logits;            /* [T,E] router logits actually used */
+  int32_t* topk_ids;        /* [T,K] original routes R_t, best first */
+  float* topk_w;            /* [T,K] original router weights */
+  float* costs;             /* [T,E] */
+  float* scores;            /* [E] */
+  int32_t* selected_ids;    /* [min(M,E)] */
+  uint8_t* active_mask;     /* [E] */
+  int32_t* exec_ids;        /* [T,K] executed routes R'_t in router-rank order, -1 = empty slot */
+  float* exec_gates;        /* [T,K] gates of the executed routes, 0 for an empty slot */
+  int32_t* expert_counts;   /* [E] tokens dispatched to each expert */
+  int32_t* n_dispatched;    /* [1] experts that received at least one token (realised active set) */
+  int32_t* status;          /* [1] OR of BASE_DEV_* bits; 0 = clean */
+} base_layer_debug;
+
+typedef struct {
+  int gate_rule;            /* BASE_GATE_* */
+  int fill_rule;            /* BASE_FILL_* */
+  int out_is_fp32;          /* 0: out is bf16 [T,d]; 1: out is fp32 [T,d] */
+  int ffn_impl;             /* 0: default (tensor-core streaming kernels); 1: simple CUDA-core kernels */
+} base_layer_options;
+
+/* Bytes of device workspace base_moe_decode_layer needs for up to T_max tokens (0 on bad shape). */
+size_t base_moe_decode_layer_workspace_bytes(const base_layer_shape* shape, int T_max);
+
+/*
+ * One BASE decode step of one MoE layer: all six steps above, enqueued on `stream`.
+ *   hidden_bf16   [T,d] bf16
+ *   router_logits [T,E] fp32 or NULL. NULL: logits = hidden . router_w^T + router_bias are computed
+ *                 here. Non-NULL: these logits are used as given (identical logits make every
+ *                 discrete routing choice reproducible between two implementations).
+ *   budget        M >= 1, clipped to E. Experts admitted but never requested receive no token and
+ *                 their weights are not read: time follows n_dispatched.
+ *   forced_mask   [E] uint8 or NULL. Non-NULL replaces the predicted selection (steps predict /
+ *                 aggregate / select still run and are reported, but routing uses this mask).
+ *   out           [T,d] bf16 or fp32 (opt->out_is_fp32)
+ *   opt, dbg      may be NULL (defaults: paper gate rule, backfill, bf16 output, default kernels)
+ *   workspace     >= base_moe_decode_layer_workspace_bytes(shape, T) bytes, 1024-byte aligned;
+ *                 contents are scratch. Calls sharing a workspace must be ordered on one stream.
+ * Limits: T <= 1024, E <= 512, K <= 16, K <= E, d % 64 == 0, I % 64 == 0 (else BASE_ERR_UNSUPPORTED).
+ */
+int base_moe_decode_layer(const base_layer_shape* shape, const base_layer_weights* weights,
+                          const void* hidden_bf16, const float* router_logits, int T, int budget,
+                          const uint8_t* forced_mask, void* out, const base_layer_options* opt,
+                          const base_layer_debug* dbg, void* workspace, size_t workspace_bytes,
+                          void* stream);
+
+/*
+ * The same step for a caller whose activations live in HOST memory: copies h_hidden_bf16 [T,d]
+ * (pinned memory recommended) into the workspace, runs the layer, copies the result to h_out and
+ * waits for `stream`. Weights stay device-resident. Needs
+ * base_moe_decode_layer_host_workspace_bytes(shape, T) bytes of device workspace.
+ * h_n_dispatched (host int32, may be NULL) receives the realised active-set size.
+ */
+size_t base_moe_decode_layer_host_workspace_bytes(const base_layer_shape* shape, int T_max);
+int base_moe_decode_layer_host(const base_layer_shape* shape, const base_layer_weights* weights,
+                               const void* h_hidden_bf16, int T, int budget, void* h_out,
+                               const base_layer_options* opt, int32_t* h_n_dispatched,
+                               void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * L layers back to back on one stream (the full-model decode-step workload). Layer l reads
+ * x_l [T,d] bf16 and the next input is x_{l+1} = rmsnorm(x_l + y_l) (no gain, fp32 math, stored
+ * bf16), which keeps inputs at unit RMS and makes the layers data dependent.
+ *   weights   HOST array of L base_layer_weights (device pointers inside)
+ *   hidden_bf16 [T,d] input of layer 0 (not modified)
+ *   out       [T,d] bf16: x_L
+ *   n_dispatched_per_layer  [L] int32 device buffer or NULL
+ * Workspace: base_moe_decode_stack_workspace_bytes(shape, T).
+ */
+size_t base_moe_decode_stack_workspace_bytes(const base_layer_shape* shape, int T_max);
+int base_moe_decode_stack(const base_layer_shape* shape, const base_layer_weights* h_weights,
+                          int L, const void* hidden_bf16, int T, int budget, void* out,
+                          const base_layer_options* opt, int32_t* n_dispatched_per_layer,
+                          void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Measurement hook (no counterpart in the paper). While a pair of cudaEvent_t handles is set for the
+ * calling thread, every layer enqueued by that thread records `start_event` on the stream just before
+ * its expert-FFN kernels and `stop_event` just after them, so a benchmark can time the dominant
+ * kernels inside a full step. Pass NULL, NULL to switch it off. Not for use during stream capture.
+ */
+int base_profile_ffn_events(void* start_event, void* stop_event);
+
+/* Number of kernels the last successful base_moe_decode_layer call on this thread enqueued. */
+int base_last_launch_count(void);
+
+const char* base_status_string(int code);
+int base_last_cuda_error(void);    /* cudaError_t of the last BASE_ERR_CUDA on this thread */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BASE_MOE_H */

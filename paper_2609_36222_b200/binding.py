@@ -1,0 +1,242 @@
+"""ctypes binding of libbase_moe.so: same names as the C ABI, argument marshalling only.
+
+Tensors are torch CUDA tensors (torch is used for device memory and streams, nothing else);
+every computation happens inside the library's kernels. There is no fallback: if the
+library is missing or a call fails, an exception is raised.
+"""
+
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libbase_moe.so")
+
+BASE_OK = 0
+GATE_PAPER, GATE_RENORM = 0, 1
+FILL_BACKFILL, FILL_DROP = 0, 1
+FFN_DEFAULT, FFN_SIMPLE = 0, 1
+DEV_NONFINITE_SCORE, DEV_WAIT_EXPIRED, DEV_BAD_INDEX = 1, 2, 4
+
+EXPORTS = (
+    "base_predict_costs", "base_aggregate_select", "base_moe_decode_layer_workspace_bytes",
+    "base_moe_decode_layer", "base_moe_decode_layer_host_workspace_bytes", "base_moe_decode_layer_host",
+    "base_moe_decode_stack_workspace_bytes", "base_moe_decode_stack", "base_profile_ffn_events",
+    "base_last_launch_count",
+    "base_status_string", "base_last_cuda_error",
+)
+
+
+class LayerShape(C.Structure):
+    _fields_ = [("d", C.c_int), ("E", C.c_int), ("K", C.c_int), ("I", C.c_int)]
+
+
+class LayerWeights(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in
+                ("router_w", "router_bias", "pred_A", "pred_b", "w_gate", "w_up", "w_down")]
+
+
+class LayerDebug(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in
+                ("logits", "topk_ids", "topk_w", "costs", "scores", "selected_ids", "active_mask",
+                 "exec_ids", "exec_gates", "expert_counts", "n_dispatched", "status")]
+
+
+class LayerOptions(C.Structure):
+    _fields_ = [("gate_rule", C.c_int), ("fill_rule", C.c_int), ("out_is_fp32", C.c_int), ("ffn_impl", C.c_int)]
+
+
+class BaseError(RuntimeError):
+    pass
+
+
+_lib = None
+
+
+def lib():
+    """Load the C-ABI library (once). Raises if it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise BaseError(f"{LIB_PATH} is missing: build it with `python -c 'import __graft_entry__ as g; g.build()'`")
+    L = C.CDLL(LIB_PATH)
+    vp, ip = C.c_void_p, C.c_int
+    L.base_predict_costs.argtypes = [vp, vp, vp, vp, vp, vp, ip, ip, ip, ip, vp]
+    L.base_aggregate_select.argtypes = [vp, ip, ip, ip, vp, vp, vp, vp]
+    L.base_moe_decode_layer_workspace_bytes.argtypes = [C.POINTER(LayerShape), ip]
+    L.base_moe_decode_layer_workspace_bytes.restype = C.c_size_t
+    L.base_moe_decode_layer.argtypes = [C.POINTER(LayerShape), C.POINTER(LayerWeights), vp, vp, ip, ip, vp, vp,
+                                        C.POINTER(LayerOptions), C.POINTER(LayerDebug), vp, C.c_size_t, vp]
+    L.base_moe_decode_layer_host_workspace_bytes.argtypes = [C.POINTER(LayerShape), ip]
+    L.base_moe_decode_layer_host_workspace_bytes.restype = C.c_size_t
+    L.base_moe_decode_layer_host.argtypes = [C.POINTER(LayerShape), C.POINTER(LayerWeights), vp, ip, ip, vp,
+                                             C.POINTER(LayerOptions), vp, vp, C.c_size_t, vp]
+    L.base_moe_decode_stack_workspace_bytes.argtypes = [C.POINTER(LayerShape), ip]
+    L.base_moe_decode_stack_workspace_bytes.restype = C.c_size_t
+    L.base_moe_decode_stack.argtypes = [C.POINTER(LayerShape), C.POINTER(LayerWeights), ip, vp, ip, ip, vp,
+                                        C.POINTER(LayerOptions), vp, vp, C.c_size_t, vp]
+    L.base_profile_ffn_events.argtypes = [vp, vp]
+    L.base_last_launch_count.restype = ip
+    L.base_status_string.argtypes = [ip]
+    L.base_status_string.restype = C.c_char_p
+    L.base_last_cuda_error.restype = ip
+    for name in EXPORTS:
+        getattr(L, name)
+        if getattr(L, name).restype is None:
+            getattr(L, name).restype = ip
+    _lib = L
+    return L
+
+
+def _check(rc):
+    if rc != BASE_OK:
+        L = lib()
+        raise BaseError(f"{L.base_status_string(rc).decode()} (code {rc}, cuda {L.base_last_cuda_error()})")
+
+
+def _ptr(t):
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    assert t.is_contiguous(), "tensors handed to the library must be contiguous"
+    return t.data_ptr()
+
+
+def _stream(stream):
+    return (stream if stream is not None else torch.cuda.current_stream()).cuda_stream
+
+
+def base_predict_costs(hidden, topk_ids, topk_w, pred_A, pred_b, costs=None, stream=None):
+    T, d = hidden.shape
+    E, K = pred_A.shape[0], topk_ids.shape[1]
+    assert hidden.dtype == torch.bfloat16 and pred_A.dtype == torch.bfloat16
+    assert topk_ids.dtype == torch.int32 and topk_w.dtype == torch.float32 and pred_b.dtype == torch.float32
+    if costs is None:
+        costs = torch.empty(T, E, dtype=torch.float32, device=hidden.device)
+    _check(lib().base_predict_costs(_ptr(hidden), _ptr(topk_ids), _ptr(topk_w), _ptr(pred_A), _ptr(pred_b),
+                                    _ptr(costs), T, d, E, K, _stream(stream)))
+    return costs
+
+
+def base_aggregate_select(costs, budget, stream=None):
+    T, E = costs.shape
+    assert costs.dtype == torch.float32
+    dev = costs.device
+    scores = torch.empty(E, dtype=torch.float32, device=dev)
+    selected = torch.full((min(budget, E),), -1, dtype=torch.int32, device=dev)
+    mask = torch.empty(E, dtype=torch.uint8, device=dev)
+    _check(lib().base_aggregate_select(_ptr(costs), T, E, budget, _ptr(scores), _ptr(selected), _ptr(mask),
+                                       _stream(stream)))
+    return scores, selected, mask
+
+
+def make_weights(tensors: dict) -> LayerWeights:
+    """tensors: router_w, router_bias, pred_A, pred_b, w_gate, w_up, w_down (torch CUDA tensors)."""
+    w = LayerWeights()
+    for name, _ in LayerWeights._fields_:
+        t = tensors.get(name)
+        if t is not None:
+            assert t.dtype == (torch.float32 if name in ("router_bias", "pred_b") else torch.bfloat16), name
+        setattr(w, name, _ptr(t))
+    return w
+
+
+DEBUG_FIELDS = {
+    "logits": ("TE", torch.float32), "topk_ids": ("TK", torch.int32), "topk_w": ("TK", torch.float32),
+    "costs": ("TE", torch.float32), "scores": ("E", torch.float32), "selected_ids": ("M", torch.int32),
+    "active_mask": ("E", torch.uint8), "exec_ids": ("TK", torch.int32), "exec_gates": ("TK", torch.float32),
+    "expert_counts": ("E", torch.int32), "n_dispatched": ("1", torch.int32), "status": ("1", torch.int32),
+}
+
+
+def alloc_debug(T, E, K, M, device):
+    """Allocate every optional intermediate buffer; returns (struct, dict of tensors)."""
+    shapes = {"TE": (T, E), "TK": (T, K), "E": (E,), "M": (min(M, E),), "1": (1,)}
+    tensors = {n: torch.zeros(shapes[s], dtype=dt, device=device) for n, (s, dt) in DEBUG_FIELDS.items()}
+    dbg = LayerDebug()
+    for n, t in tensors.items():
+        setattr(dbg, n, _ptr(t))
+    return dbg, tensors
+
+
+def layer_workspace_bytes(d, E, K, I, T_max):
+    n = lib().base_moe_decode_layer_workspace_bytes(C.byref(LayerShape(d, E, K, I)), T_max)
+    if n == 0:
+        raise BaseError("unsupported shape")
+    return n
+
+
+def alloc_workspace(nbytes, device):
+    """1024-byte aligned device buffer."""
+    buf = torch.empty(nbytes + 1024, dtype=torch.uint8, device=device)
+    off = (-buf.data_ptr()) % 1024
+    return buf[off:off + nbytes]
+
+
+def base_moe_decode_layer(shape, weights, hidden, budget, out, workspace, router_logits=None, forced_mask=None,
+                          gate_rule=GATE_PAPER, fill_rule=FILL_BACKFILL, ffn_impl=FFN_DEFAULT, debug=None,
+                          stream=None):
+    """shape: (d, E, K, I); weights: LayerWeights; out: [T,d] bf16 or fp32 tensor (written in place)."""
+    d, E, K, I = shape
+    T = hidden.shape[0]
+    assert hidden.dtype == torch.bfloat16 and hidden.shape[1] == d
+    assert out.dtype in (torch.bfloat16, torch.float32) and tuple(out.shape) == (T, d)
+    if router_logits is not None:
+        assert router_logits.dtype == torch.float32 and tuple(router_logits.shape) == (T, E)
+    if forced_mask is not None:
+        assert forced_mask.dtype == torch.uint8 and forced_mask.numel() == E
+    opt = LayerOptions(gate_rule, fill_rule, 1 if out.dtype == torch.float32 else 0, ffn_impl)
+    _check(lib().base_moe_decode_layer(C.byref(LayerShape(d, E, K, I)), C.byref(weights), _ptr(hidden),
+                                       _ptr(router_logits), T, budget, _ptr(forced_mask), _ptr(out), C.byref(opt),
+                                       C.byref(debug) if debug is not None else None, _ptr(workspace),
+                                       workspace.numel(), _stream(stream)))
+    return out
+
+
+def layer_host_workspace_bytes(d, E, K, I, T_max):
+    n = lib().base_moe_decode_layer_host_workspace_bytes(C.byref(LayerShape(d, E, K, I)), T_max)
+    if n == 0:
+        raise BaseError("unsupported shape")
+    return n
+
+
+def base_moe_decode_layer_host(shape, weights, h_hidden, budget, h_out, workspace, gate_rule=GATE_PAPER,
+                               fill_rule=FILL_BACKFILL, ffn_impl=FFN_DEFAULT, h_n_dispatched=None, stream=None):
+    """h_hidden / h_out: CPU (preferably pinned) torch tensors; blocks until h_out is written."""
+    d, E, K, I = shape
+    T = h_hidden.shape[0]
+    assert not h_hidden.is_cuda and not h_out.is_cuda and h_hidden.dtype == torch.bfloat16
+    opt = LayerOptions(gate_rule, fill_rule, 1 if h_out.dtype == torch.float32 else 0, ffn_impl)
+    _check(lib().base_moe_decode_layer_host(C.byref(LayerShape(d, E, K, I)), C.byref(weights), _ptr(h_hidden), T,
+                                            budget, _ptr(h_out), C.byref(opt), _ptr(h_n_dispatched), _ptr(workspace),
+                                            workspace.numel(), _stream(stream)))
+    return h_out
+
+
+def stack_workspace_bytes(d, E, K, I, T_max):
+    n = lib().base_moe_decode_stack_workspace_bytes(C.byref(LayerShape(d, E, K, I)), T_max)
+    if n == 0:
+        raise BaseError("unsupported shape")
+    return n
+
+
+def base_moe_decode_stack(shape, weights_list, hidden, budget, out, workspace, n_dispatched=None,
+                          gate_rule=GATE_PAPER, fill_rule=FILL_BACKFILL, ffn_impl=FFN_DEFAULT, stream=None):
+    d, E, K, I = shape
+    T = hidden.shape[0]
+    L = len(weights_list)
+    arr = (LayerWeights * L)(*weights_list)
+    opt = LayerOptions(gate_rule, fill_rule, 0, ffn_impl)
+    _check(lib().base_moe_decode_stack(C.byref(LayerShape(d, E, K, I)), arr, L, _ptr(hidden), T, budget, _ptr(out),
+                                       C.byref(opt), _ptr(n_dispatched), _ptr(workspace), workspace.numel(),
+                                       _stream(stream)))
+    return out
+
+
+def last_launch_count():
+    return lib().base_last_launch_count()

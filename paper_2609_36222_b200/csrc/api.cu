@@ -1,0 +1,276 @@
+// C-ABI entry points: argument checks, workspace carving, kernel sequencing. No device allocation,
+// no synchronisation (except the *_host entry point, which waits for its own copies).
+#include <string.h>
+
+#include "common.cuh"
+#include "ffn_tc.cuh"
+
+using namespace base;
+
+namespace {
+
+thread_local int g_last_cuda_error = 0;
+thread_local int g_last_launches = 0;
+thread_local cudaEvent_t g_ev_start = nullptr, g_ev_stop = nullptr;
+
+inline int cuda_fail(cudaError_t e) {
+  g_last_cuda_error = int(e);
+  return BASE_ERR_CUDA;
+}
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_shape(const base_layer_shape* s, int T) {
+  if (!s || s->d <= 0 || s->E <= 0 || s->K <= 0 || s->I <= 0 || T <= 0) return BASE_ERR_INVALID_ARG;
+  if (s->K > s->E) return BASE_ERR_INVALID_ARG;
+  if (T > kMaxT || s->E > kMaxE || s->K > kMaxK || size_t(T) * s->K > size_t(kMaxSlots)) return BASE_ERR_UNSUPPORTED;
+  if (s->d % 64 != 0 || s->I % 64 != 0 || s->d > 8192) return BASE_ERR_UNSUPPORTED;
+  return BASE_OK;
+}
+
+struct LayerCall {
+  const base_layer_shape* shape;
+  const base_layer_weights* w;
+  const void* hidden;
+  const float* router_logits;
+  int T, budget;
+  const uint8_t* forced_mask;
+  void* out;
+  base_layer_options opt;
+  base_layer_debug dbg;
+  void* x_next;  // stack wiring output or nullptr
+};
+
+// Enqueue one layer on `st` using an already carved workspace.
+int enqueue_layer(const LayerCall& c, const Workspace& ws, cudaStream_t st, int* launches) {
+  const base_layer_shape& s = *c.shape;
+  cudaError_t e;
+  const float* logits = c.router_logits;
+  e = launch_route_scores(c.hidden, c.w->router_w, c.w->router_bias, c.w->pred_A, c.w->pred_b,
+                          logits ? nullptr : ws.logits, ws.shat, c.T, s.d, s.E, st);
+  if (e != cudaSuccess) return cuda_fail(e);
+  ++*launches;
+  if (!logits) logits = ws.logits;
+
+  RoutingArgs ra{};
+  ra.logits = logits;
+  ra.shat = ws.shat;
+  ra.forced_mask = c.forced_mask;
+  ra.T = c.T;
+  ra.E = s.E;
+  ra.K = s.K;
+  ra.M = c.budget;
+  ra.gate_rule = c.opt.gate_rule;
+  ra.fill_rule = c.opt.fill_rule;
+  ra.ws = ws;
+  ra.dbg = c.dbg;
+  e = launch_routing(ra, st);
+  if (e != cudaSuccess) return cuda_fail(e);
+  ++*launches;
+
+  e = launch_gather(c.hidden, ws, c.T, s.K, s.d, st);
+  if (e != cudaSuccess) return cuda_fail(e);
+  ++*launches;
+
+  if (g_ev_start) cudaEventRecord(g_ev_start, st);
+  if (c.opt.ffn_impl == 1) {
+    e = launch_ffn_simple(s, *c.w, ws, st, launches);
+  } else {
+    e = launch_ffn_tc(s, *c.w, ws, c.T, st, launches);
+  }
+  if (e != cudaSuccess) return cuda_fail(e);
+  if (g_ev_stop) cudaEventRecord(g_ev_stop, st);
+
+  e = launch_combine(ws, c.hidden, c.out, c.opt.out_is_fp32, c.x_next, c.T, s.K, s.d, st);
+  if (e != cudaSuccess) return cuda_fail(e);
+  ++*launches;
+  return BASE_OK;
+}
+
+int check_layer_args(const base_layer_shape* shape, const base_layer_weights* w, const void* hidden,
+                     const float* router_logits, int T, int budget, const base_layer_options* opt) {
+  int rc = check_shape(shape, T);
+  if (rc != BASE_OK) return rc;
+  if (!w || !hidden || budget <= 0) return BASE_ERR_INVALID_ARG;
+  if (!w->pred_A || !w->pred_b || !w->w_gate || !w->w_up || !w->w_down) return BASE_ERR_INVALID_ARG;
+  if (!router_logits && !w->router_w) return BASE_ERR_INVALID_ARG;
+  if (!aligned16(hidden) || !aligned16(w->pred_A) || !aligned16(w->w_gate) || !aligned16(w->w_up) ||
+      !aligned16(w->w_down) || (w->router_w && !aligned16(w->router_w)))
+    return BASE_ERR_INVALID_ARG;
+  if (opt) {
+    if (opt->gate_rule != BASE_GATE_PAPER && opt->gate_rule != BASE_GATE_RENORM) return BASE_ERR_INVALID_ARG;
+    if (opt->fill_rule != BASE_FILL_BACKFILL && opt->fill_rule != BASE_FILL_DROP) return BASE_ERR_INVALID_ARG;
+    if (opt->ffn_impl != 0 && opt->ffn_impl != 1) return BASE_ERR_INVALID_ARG;
+  }
+  return BASE_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int base_predict_costs(const void* hidden_bf16, const int32_t* topk_ids, const float* topk_w,
+                       const void* pred_A_bf16, const float* pred_b, float* costs, int T, int d, int E, int K,
+                       void* stream) {
+  if (!hidden_bf16 || !topk_ids || !topk_w || !pred_A_bf16 || !pred_b || !costs) return BASE_ERR_INVALID_ARG;
+  if (T <= 0 || d <= 0 || E <= 0 || K <= 0) return BASE_ERR_INVALID_ARG;
+  if (!aligned16(hidden_bf16) || !aligned16(pred_A_bf16)) return BASE_ERR_INVALID_ARG;
+  if (d % 8 != 0 || K > 64) return BASE_ERR_UNSUPPORTED;
+  cudaError_t e = launch_predict_costs(hidden_bf16, topk_ids, topk_w, pred_A_bf16, pred_b, costs, T, d, E, K,
+                                       static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? BASE_OK : cuda_fail(e);
+}
+
+int base_aggregate_select(const float* costs, int T, int E, int budget, float* scores, int32_t* selected_ids,
+                          uint8_t* active_mask, void* stream) {
+  if (!costs || !scores || !selected_ids || !active_mask) return BASE_ERR_INVALID_ARG;
+  if (T <= 0 || E <= 0 || budget <= 0) return BASE_ERR_INVALID_ARG;
+  if (E > 1024) return BASE_ERR_UNSUPPORTED;
+  cudaError_t e = launch_aggregate_select(costs, T, E, budget < E ? budget : E, scores, selected_ids, active_mask,
+                                          static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? BASE_OK : cuda_fail(e);
+}
+
+size_t base_moe_decode_layer_workspace_bytes(const base_layer_shape* shape, int T_max) {
+  if (check_shape(shape, T_max) != BASE_OK) return 0;
+  return carve_workspace(nullptr, *shape, T_max).bytes;
+}
+
+int base_moe_decode_layer(const base_layer_shape* shape, const base_layer_weights* weights, const void* hidden_bf16,
+                          const float* router_logits, int T, int budget, const uint8_t* forced_mask, void* out,
+                          const base_layer_options* opt, const base_layer_debug* dbg, void* workspace,
+                          size_t workspace_bytes, void* stream) {
+  int rc = check_layer_args(shape, weights, hidden_bf16, router_logits, T, budget, opt);
+  if (rc != BASE_OK) return rc;
+  if (!out || !workspace || !aligned16(out)) return BASE_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(workspace) & 1023u) return BASE_ERR_INVALID_ARG;
+  Workspace ws = carve_workspace(workspace, *shape, T);
+  if (ws.bytes > workspace_bytes) return BASE_ERR_WORKSPACE_TOO_SMALL;
+  LayerCall c{};
+  c.shape = shape;
+  c.w = weights;
+  c.hidden = hidden_bf16;
+  c.router_logits = router_logits;
+  c.T = T;
+  c.budget = budget;
+  c.forced_mask = forced_mask;
+  c.out = out;
+  if (opt) c.opt = *opt;
+  if (dbg) c.dbg = *dbg;
+  int launches = 0;
+  rc = enqueue_layer(c, ws, static_cast<cudaStream_t>(stream), &launches);
+  if (rc == BASE_OK) g_last_launches = launches;
+  return rc;
+}
+
+size_t base_moe_decode_layer_host_workspace_bytes(const base_layer_shape* shape, int T_max) {
+  if (check_shape(shape, T_max) != BASE_OK) return 0;
+  const size_t io = align_up(size_t(T_max) * shape->d * 2, 1024) + align_up(size_t(T_max) * shape->d * 4, 1024) + 1024;
+  return carve_workspace(nullptr, *shape, T_max).bytes + io;
+}
+
+int base_moe_decode_layer_host(const base_layer_shape* shape, const base_layer_weights* weights,
+                               const void* h_hidden_bf16, int T, int budget, void* h_out,
+                               const base_layer_options* opt, int32_t* h_n_dispatched, void* workspace,
+                               size_t workspace_bytes, void* stream) {
+  int rc = check_layer_args(shape, weights, h_hidden_bf16, nullptr, T, budget, opt);
+  if (rc != BASE_OK) return rc;
+  if (!h_out || !workspace || (reinterpret_cast<uintptr_t>(workspace) & 1023u)) return BASE_ERR_INVALID_ARG;
+  if (base_moe_decode_layer_host_workspace_bytes(shape, T) > workspace_bytes) return BASE_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  Workspace ws = carve_workspace(workspace, *shape, T);
+  char* io = static_cast<char*>(workspace) + ws.bytes;
+  void* d_in = io;
+  void* d_out = io + align_up(size_t(T) * shape->d * 2, 1024);
+  int32_t* d_nd = reinterpret_cast<int32_t*>(static_cast<char*>(d_out) + align_up(size_t(T) * shape->d * 4, 1024));
+  cudaError_t e = cudaMemcpyAsync(d_in, h_hidden_bf16, size_t(T) * shape->d * 2, cudaMemcpyHostToDevice, st);
+  if (e != cudaSuccess) return cuda_fail(e);
+  LayerCall c{};
+  c.shape = shape;
+  c.w = weights;
+  c.hidden = d_in;
+  c.T = T;
+  c.budget = budget;
+  c.out = d_out;
+  if (opt) c.opt = *opt;
+  c.dbg.n_dispatched = d_nd;
+  int launches = 0;
+  rc = enqueue_layer(c, ws, st, &launches);
+  if (rc != BASE_OK) return rc;
+  const size_t out_bytes = size_t(T) * shape->d * (c.opt.out_is_fp32 ? 4 : 2);
+  e = cudaMemcpyAsync(h_out, d_out, out_bytes, cudaMemcpyDeviceToHost, st);
+  if (e != cudaSuccess) return cuda_fail(e);
+  if (h_n_dispatched) {
+    e = cudaMemcpyAsync(h_n_dispatched, d_nd, 4, cudaMemcpyDeviceToHost, st);
+    if (e != cudaSuccess) return cuda_fail(e);
+  }
+  e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess) return cuda_fail(e);
+  g_last_launches = launches;
+  return BASE_OK;
+}
+
+size_t base_moe_decode_stack_workspace_bytes(const base_layer_shape* shape, int T_max) {
+  if (check_shape(shape, T_max) != BASE_OK) return 0;
+  return carve_workspace(nullptr, *shape, T_max).bytes + 2 * align_up(size_t(T_max) * shape->d * 2, 1024);
+}
+
+int base_moe_decode_stack(const base_layer_shape* shape, const base_layer_weights* h_weights, int L,
+                          const void* hidden_bf16, int T, int budget, void* out, const base_layer_options* opt,
+                          int32_t* n_dispatched_per_layer, void* workspace, size_t workspace_bytes, void* stream) {
+  if (L <= 0 || !h_weights) return BASE_ERR_INVALID_ARG;
+  for (int l = 0; l < L; ++l) {
+    int rc = check_layer_args(shape, &h_weights[l], hidden_bf16, nullptr, T, budget, opt);
+    if (rc != BASE_OK) return rc;
+  }
+  if (!out || !workspace || !aligned16(out) || (reinterpret_cast<uintptr_t>(workspace) & 1023u))
+    return BASE_ERR_INVALID_ARG;
+  if (base_moe_decode_stack_workspace_bytes(shape, T) > workspace_bytes) return BASE_ERR_WORKSPACE_TOO_SMALL;
+  Workspace ws = carve_workspace(workspace, *shape, T);
+  char* extra = static_cast<char*>(workspace) + ws.bytes;
+  void* ping[2] = {extra, extra + align_up(size_t(T) * shape->d * 2, 1024)};
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int launches = 0;
+  const void* x = hidden_bf16;
+  for (int l = 0; l < L; ++l) {
+    LayerCall c{};
+    c.shape = shape;
+    c.w = &h_weights[l];
+    c.hidden = x;
+    c.T = T;
+    c.budget = budget;
+    c.out = nullptr;  // only the wired next input is needed
+    if (opt) c.opt = *opt;
+    if (n_dispatched_per_layer) c.dbg.n_dispatched = n_dispatched_per_layer + l;
+    c.x_next = (l == L - 1) ? out : ping[l & 1];
+    int rc = enqueue_layer(c, ws, st, &launches);
+    if (rc != BASE_OK) return rc;
+    x = c.x_next;
+  }
+  g_last_launches = launches;
+  return BASE_OK;
+}
+
+int base_profile_ffn_events(void* start_event, void* stop_event) {
+  if ((start_event == nullptr) != (stop_event == nullptr)) return BASE_ERR_INVALID_ARG;
+  g_ev_start = static_cast<cudaEvent_t>(start_event);
+  g_ev_stop = static_cast<cudaEvent_t>(stop_event);
+  return BASE_OK;
+}
+
+int base_last_launch_count(void) { return g_last_launches; }
+
+const char* base_status_string(int code) {
+  switch (code) {
+    case BASE_OK: return "ok";
+    case BASE_ERR_INVALID_ARG: return "invalid argument";
+    case BASE_ERR_UNSUPPORTED: return "shape outside the compiled limits";
+    case BASE_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case BASE_ERR_CUDA: return "CUDA error (see base_last_cuda_error)";
+    default: return "unknown status";
+  }
+}
+
+int base_last_cuda_error(void) { return g_last_cuda_error; }
+
+}  // extern "C"

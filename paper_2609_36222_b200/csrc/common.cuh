@@ -1,0 +1,145 @@
+// Shared device helpers and the workspace layout of the decode layer (sm_100a only).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "base_moe.h"
+
+namespace base {
+
+constexpr int kWarp = 32;
+constexpr int kMaxE = 512;          // experts per layer (routing kernel keeps E/32 logits per lane)
+constexpr int kMaxVals = kMaxE / kWarp;
+constexpr int kMaxK = 16;
+constexpr int kMaxT = 1024;
+constexpr int kMaxSlots = 8192;     // T*K routed pairs held in shared memory by the routing kernel
+constexpr int kSegTokens = 128;     // tokens of one expert handled by one FFN work unit
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+// Eight bf16 values packed in a uint4 -> fp32.
+__device__ __forceinline__ void unpack8(const uint4& v, float (&f)[8]) {
+  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    f[2 * i] = __uint_as_float(w[i] << 16);
+    f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+  }
+}
+
+__device__ __forceinline__ uint4 ldg16(const void* p) { return __ldg(reinterpret_cast<const uint4*>(p)); }
+
+__device__ __forceinline__ float silu_f(float x) { return x / (1.0f + expf(-x)); }
+
+// Pointers into the caller's workspace for one layer call (all device memory).
+struct Workspace {
+  float* logits;          // [T,E]
+  float* shat;            // [T,E] predicted log-energy of every (token, expert) pair
+  float* costs;           // [T,E]
+  int32_t* topk_ids;      // [T,K]
+  float* topk_w;          // [T,K]
+  float* scores;          // [E]
+  int32_t* selected;      // [E]
+  uint8_t* mask;          // [E] predicted active set
+  int32_t* exec_ids;      // [T,K]
+  float* exec_gates;      // [T,K]
+  int32_t* token_slot;    // [T,K] row of (t,k) in the expert-sorted buffers, -1 = empty
+  int32_t* slot_token;    // [T*K]
+  int32_t* expert_count;  // [E]
+  int32_t* expert_offset; // [E+1]
+  int32_t* seg_expert;    // [max_segs] work segments: one expert, at most kSegTokens tokens
+  int32_t* seg_offset;    // [max_segs] first sorted row of the segment
+  int32_t* seg_count;     // [max_segs]
+  int32_t* counters;      // [16 + E]: 0 n_dispatched, 1 n_segments, 2 status, 3 total slots, 4.. tickets; 16.. per-expert ready
+  __nv_bfloat16* x_sorted; // [T*K + pad, d] token inputs in expert-sorted order
+  __nv_bfloat16* h;        // [T*K + pad, I] silu(gate) * up, expert-sorted
+  float* ypair;            // [T*K, d] down-projection outputs per routed pair
+  __nv_bfloat16* x_next;   // [T,d] scratch for the stack / host entry points
+  size_t bytes;
+};
+
+constexpr int kCtrDispatched = 0, kCtrSegments = 1, kCtrStatus = 2, kCtrSlots = 3, kCtrTicket = 4, kCtrReady = 16;
+constexpr int kRowPad = 256;  // rows readable past the last sorted row (tile over-read stays in bounds)
+
+inline int max_segments(int E, int T, int K) { return E + (T * K) / kSegTokens + 1; }
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Carve the workspace. With base == nullptr only the size is computed.
+inline Workspace carve_workspace(void* base_ptr, const base_layer_shape& s, int T) {
+  Workspace w{};
+  size_t off = 0;
+  char* b = static_cast<char*>(base_ptr);
+  auto take = [&](size_t bytes, size_t align) -> void* {
+    off = align_up(off, align);
+    void* p = b ? b + off : nullptr;
+    off += bytes;
+    return p;
+  };
+  const size_t TE = size_t(T) * s.E, TK = size_t(T) * s.K;
+  const int segs = max_segments(s.E, T, s.K);
+  w.x_sorted = static_cast<__nv_bfloat16*>(take((TK + kRowPad) * s.d * 2, 1024));
+  w.h = static_cast<__nv_bfloat16*>(take((TK + kRowPad) * s.I * 2, 1024));
+  w.ypair = static_cast<float*>(take(TK * s.d * 4, 1024));
+  w.x_next = static_cast<__nv_bfloat16*>(take(size_t(T) * s.d * 2, 1024));
+  w.logits = static_cast<float*>(take(TE * 4, 256));
+  w.shat = static_cast<float*>(take(TE * 4, 256));
+  w.costs = static_cast<float*>(take(TE * 4, 256));
+  w.topk_ids = static_cast<int32_t*>(take(TK * 4, 256));
+  w.topk_w = static_cast<float*>(take(TK * 4, 256));
+  w.scores = static_cast<float*>(take(size_t(s.E) * 4, 256));
+  w.selected = static_cast<int32_t*>(take(size_t(s.E) * 4, 256));
+  w.mask = static_cast<uint8_t*>(take(size_t(s.E), 256));
+  w.exec_ids = static_cast<int32_t*>(take(TK * 4, 256));
+  w.exec_gates = static_cast<float*>(take(TK * 4, 256));
+  w.token_slot = static_cast<int32_t*>(take(TK * 4, 256));
+  w.slot_token = static_cast<int32_t*>(take(TK * 4, 256));
+  w.expert_count = static_cast<int32_t*>(take(size_t(s.E) * 4, 256));
+  w.expert_offset = static_cast<int32_t*>(take(size_t(s.E + 1) * 4, 256));
+  w.seg_expert = static_cast<int32_t*>(take(size_t(segs) * 4, 256));
+  w.seg_offset = static_cast<int32_t*>(take(size_t(segs) * 4, 256));
+  w.seg_count = static_cast<int32_t*>(take(size_t(segs) * 4, 256));
+  w.counters = static_cast<int32_t*>(take(size_t(kCtrReady + s.E) * 4, 256));
+  w.bytes = align_up(off, 1024);
+  return w;
+}
+
+// ---- host-side launchers implemented in the .cu files (return cudaGetLastError of the launch) ----
+
+struct RoutingArgs {
+  const float* logits;        // [T,E] logits to route on
+  const float* shat;          // [T,E]
+  const uint8_t* forced_mask; // or nullptr
+  int T, E, K, M, gate_rule, fill_rule;
+  Workspace ws;
+  base_layer_debug dbg;       // zero-initialised when the caller passed none
+};
+
+cudaError_t launch_predict_costs(const void* hidden, const int32_t* ids, const float* w, const void* A,
+                                 const float* b, float* costs, int T, int d, int E, int K, cudaStream_t st);
+cudaError_t launch_aggregate_select(const float* costs, int T, int E, int M, float* scores, int32_t* sel,
+                                    uint8_t* mask, cudaStream_t st);
+cudaError_t launch_route_scores(const void* hidden, const void* router_w, const float* router_bias,
+                                const void* pred_A, const float* pred_b, float* logits_out, float* shat,
+                                int T, int d, int E, cudaStream_t st);
+cudaError_t launch_routing(const RoutingArgs& a, cudaStream_t st);
+cudaError_t launch_gather(const void* hidden, const Workspace& ws, int T, int K, int d, cudaStream_t st);
+cudaError_t launch_combine(const Workspace& ws, const void* hidden, void* out, int out_is_fp32, void* x_next,
+                           int T, int K, int d, cudaStream_t st);
+
+cudaError_t launch_ffn_simple(const base_layer_shape& s, const base_layer_weights& w, const Workspace& ws,
+                              cudaStream_t st, int* launches);
+
+}  // namespace base

@@ -1,0 +1,49 @@
+"""Convenience holder for one layer's device tensors and workspace (memory plumbing only)."""
+
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from . import binding as B
+from . import workloads as wl
+
+
+def bits_to_device(bits: np.ndarray, device) -> torch.Tensor:
+    """uint16 bf16 bit patterns (host) -> bf16 tensor on the device."""
+    return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).to(device).view(torch.bfloat16)
+
+
+class DeviceLayer:
+    """Weights of one synthetic layer resident on the device, plus a workspace for up to T_max tokens."""
+
+    def __init__(self, cfg: wl.LayerConfig, device, seed: int = 0, layer: int = 0, T_max: int | None = None,
+                 small: dict | None = None, expert_bits: dict | None = None, workspace=None):
+        self.cfg, self.device = cfg, device
+        self.shape = (cfg.d, cfg.E, cfg.K, cfg.I)
+        small = small if small is not None else wl.small_tensors(cfg, seed, layer)
+        self.tensors = {
+            "router_w": bits_to_device(small["router_w"], device),
+            "pred_A": bits_to_device(small["pred_A"], device),
+            "router_bias": torch.from_numpy(small["router_bias"]).to(device),
+            "pred_b": torch.from_numpy(small["pred_b"]).to(device),
+        }
+        if expert_bits is not None:
+            for k, v in expert_bits.items():
+                self.tensors[k] = bits_to_device(v, device)
+        else:
+            self.tensors.update(wl.expert_weights_device(cfg, device, seed, layer))
+        self.weights = B.make_weights(self.tensors)
+        self.T_max = T_max if T_max is not None else cfg.T
+        self.workspace = workspace if workspace is not None else B.alloc_workspace(
+            B.layer_workspace_bytes(*self.shape, self.T_max), device)
+
+    def set_predictor(self, A_bits: np.ndarray, b: np.ndarray):
+        self.tensors["pred_A"] = bits_to_device(A_bits, self.device)
+        self.tensors["pred_b"] = torch.from_numpy(np.ascontiguousarray(b, dtype=np.float32)).to(self.device)
+        self.weights = B.make_weights(self.tensors)
+
+    def run(self, hidden: torch.Tensor, budget: int, out: torch.Tensor | None = None, **kw) -> torch.Tensor:
+        if out is None:
+            out = torch.empty(hidden.shape[0], self.cfg.d, dtype=torch.bfloat16, device=self.device)
+        return B.base_moe_decode_layer(self.shape, self.weights, hidden, budget, out, self.workspace, **kw)

@@ -138,7 +138,21 @@ def _bf16_table(sigma: float) -> np.ndarray:
 
 
 def _index_np(key: int, start: int, count: int) -> np.ndarray:
-    return (mix64_np(key, start, count) >> np.uint64(64 - TABLE_BITS)).astype(np.int64)
+    """Table indices (top 16 bits of the stream), computed in place on one temporary."""
+    with np.errstate(over="ignore"):
+        z = np.arange(start + 1, start + 1 + count, dtype=np.uint64)
+        z *= np.uint64(_GAMMA)
+        z += np.uint64(key)
+        t = z >> np.uint64(30)
+        z ^= t
+        z *= np.uint64(_M1)
+        np.right_shift(z, np.uint64(27), out=t)
+        z ^= t
+        z *= np.uint64(_M2)
+        np.right_shift(z, np.uint64(31), out=t)
+        z ^= t
+        z >>= np.uint64(64 - TABLE_BITS)
+    return z
 
 
 def normal_f64(key: int, start: int, count: int) -> np.ndarray:
@@ -146,13 +160,25 @@ def normal_f64(key: int, start: int, count: int) -> np.ndarray:
     return normal_quantiles()[_index_np(key, start, count)]
 
 
-def normal_bf16_bits(key: int, start: int, count: int, sigma: float, chunk: int = 1 << 24) -> np.ndarray:
-    """N(0, sigma) draws rounded to bf16, as uint16 bit patterns (host)."""
+def normal_bf16_bits(key: int, start: int, count: int, sigma: float, chunk: int = 1 << 18,
+                     threads: int | None = None) -> np.ndarray:
+    """N(0, sigma) draws rounded to bf16, as uint16 bit patterns (host; chunks run on a thread pool)."""
     table = _bf16_table(float(sigma))
     out = np.empty(count, dtype=np.uint16)
-    for off in range(0, count, chunk):
+
+    def work(off):
         n = min(chunk, count - off)
         out[off:off + n] = table[_index_np(key, start + off, n)]
+
+    offsets = range(0, count, chunk)
+    if count <= chunk:
+        for off in offsets:
+            work(off)
+    else:
+        from concurrent.futures import ThreadPoolExecutor
+        import os
+        with ThreadPoolExecutor(threads or min(16, os.cpu_count() or 1)) as ex:
+            list(ex.map(work, offsets))
     return out
 
 

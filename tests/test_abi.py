@@ -1,0 +1,70 @@
+"""The C-ABI library builds, loads, exports every symbol the header declares, and rejects bad
+arguments before touching the device (no GPU needed)."""
+
+import ctypes as C
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    import __graft_entry__ as g
+    g.build()
+    from paper_2609_36222_b200 import binding as B
+    return B.lib()
+
+
+def declared_functions():
+    names = set()
+    for fn in os.listdir(os.path.join(ROOT, "include")):
+        if fn.endswith(".h"):
+            text = open(os.path.join(ROOT, "include", fn)).read()
+            text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+            names |= set(re.findall(r"\b(base_[a-z0-9_]+)\s*\(", text))
+    return names
+
+
+def test_every_declared_symbol_is_exported(lib):
+    from paper_2609_36222_b200 import binding as B
+    names = declared_functions()
+    assert {"base_predict_costs", "base_aggregate_select", "base_moe_decode_layer"} <= names
+    raw = C.CDLL(B.LIB_PATH)
+    for n in names:
+        assert getattr(raw, n) is not None, n
+    assert names == set(B.EXPORTS)
+
+
+def test_status_strings(lib):
+    for code, word in [(0, "ok"), (1, "invalid"), (2, "limits"), (3, "workspace"), (4, "CUDA")]:
+        assert word in lib.base_status_string(code).decode()
+    assert "unknown" in lib.base_status_string(99).decode()
+
+
+def test_argument_checks_need_no_device(lib):
+    from paper_2609_36222_b200 import binding as B
+    assert lib.base_predict_costs(None, None, None, None, None, None, 1, 8, 1, 1, None) == 1
+    assert lib.base_aggregate_select(None, 1, 1, 1, None, None, None, None) == 1
+    assert lib.base_aggregate_select(16, 4, 2000, 1, 16, 16, 16, None) == 2
+    ok = B.LayerShape(2048, 128, 8, 768)
+    assert lib.base_moe_decode_layer_workspace_bytes(C.byref(ok), 64) > 64 * 8 * 2048 * 4
+    assert lib.base_moe_decode_layer_workspace_bytes(C.byref(B.LayerShape(2040, 128, 8, 768)), 64) == 0
+    assert lib.base_moe_decode_layer_workspace_bytes(C.byref(B.LayerShape(2048, 4, 8, 768)), 64) == 0
+    assert lib.base_moe_decode_layer_workspace_bytes(C.byref(ok), 5000) == 0
+    w = B.LayerWeights()
+    assert lib.base_moe_decode_layer(C.byref(ok), C.byref(w), 16, None, 4, 2, None, 16, None, None, 1024, 1 << 30,
+                                     None) == 1      # null weights
+    big = lib.base_moe_decode_layer_host_workspace_bytes(C.byref(ok), 64)
+    assert big > lib.base_moe_decode_layer_workspace_bytes(C.byref(ok), 64)
+    assert lib.base_moe_decode_stack_workspace_bytes(C.byref(ok), 64) > 0
+
+
+def test_binding_fails_loudly_without_library(monkeypatch, tmp_path):
+    from paper_2609_36222_b200 import binding as B
+    monkeypatch.setattr(B, "_lib", None)
+    monkeypatch.setattr(B, "LIB_PATH", str(tmp_path / "missing.so"))
+    with pytest.raises(B.BaseError, match="missing"):
+        B.lib()
