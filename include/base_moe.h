@@ -140,7 +140,8 @@ size_t base_moe_decode_layer_workspace_bytes(const base_layer_shape* shape, int 
  *   opt, dbg      may be NULL (defaults: paper gate rule, backfill, bf16 output, default kernels)
  *   workspace     >= base_moe_decode_layer_workspace_bytes(shape, T) bytes, 1024-byte aligned;
  *                 contents are scratch. Calls sharing a workspace must be ordered on one stream.
- * Limits: T <= 1024, E <= 512, K <= 16, K <= E, d % 64 == 0, I % 64 == 0 (else BASE_ERR_UNSUPPORTED).
+ * Limits: T <= 1024, T*K <= 8192, E <= 512, K <= 16, K <= E, d <= 8192, d % 128 == 0 (d % 64 == 0 with the
+ * simple kernels), I % 64 == 0 (else BASE_ERR_UNSUPPORTED).
  */
 int base_moe_decode_layer(const base_layer_shape* shape, const base_layer_weights* weights,
                           const void* hidden_bf16, const float* router_logits, int T, int budget,

@@ -97,6 +97,7 @@ int check_layer_args(const base_layer_shape* shape, const base_layer_weights* w,
   if (!aligned16(hidden) || !aligned16(w->pred_A) || !aligned16(w->w_gate) || !aligned16(w->w_up) ||
       !aligned16(w->w_down) || (w->router_w && !aligned16(w->router_w)))
     return BASE_ERR_INVALID_ARG;
+  if ((!opt || opt->ffn_impl == 0) && shape->d % 128 != 0) return BASE_ERR_UNSUPPORTED;
   if (opt) {
     if (opt->gate_rule != BASE_GATE_PAPER && opt->gate_rule != BASE_GATE_RENORM) return BASE_ERR_INVALID_ARG;
     if (opt->fill_rule != BASE_FILL_BACKFILL && opt->fill_rule != BASE_FILL_DROP) return BASE_ERR_INVALID_ARG;

@@ -207,7 +207,7 @@ def test_error_codes(layers):
     with pytest.raises(B.BaseError, match="workspace"):
         B.base_moe_decode_layer(dl.shape, dl.weights, hid, 4, out, dl.workspace[:1024])
     with pytest.raises(B.BaseError, match="limits"):
-        B.base_moe_decode_layer((250, 16, 4, 128), dl.weights, hid, 4, out, dl.workspace)
+        B.base_moe_decode_layer((256, 16, 4, 100), dl.weights, hid, 4, out, dl.workspace)
     with pytest.raises(B.BaseError, match="invalid"):
         B.base_moe_decode_layer(dl.shape, dl.weights, hid, 4, out, dl.workspace, gate_rule=7)
 
