@@ -272,7 +272,7 @@ def run_ours(args, cfg, T, M):
     with ClockSampler(local) as clocks:
         ms = timed(graphs, args.steps, args.warmup)
         # keep the sampler alive long enough to see the load when the run is very short
-        if ms * args.steps < 300:
+        if ms * args.steps < 300 and not args.profile:
             timed(graphs, max(args.steps, int(300 / max(ms, 1e-3))), 0)
     clk = clocks.summary()
     if dist is not None:
@@ -282,25 +282,27 @@ def run_ours(args, cfg, T, M):
 
     # ---- per-kernel pass for the roofline: the library records the caller's events around the FFN kernels
     n_prof = min(args.steps, 40)
-    ffn_us = None
-    if hasattr(B.lib(), "base_profile_ffn_events"):
-        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_prof)]
+    ffn_us, stage_us = None, None
+    if not args.profile:
+        evs = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(n_prof)]
         with torch.cuda.stream(stream):
             for i in range(3):
                 step_eager(i)
-            for i, (a, b) in enumerate(evs):
-                a.record(stream)   # create both handles before the library records them again
-                b.record(stream)
-                B.lib().base_profile_ffn_events(a.cuda_event, b.cuda_event)
+            for i, ev in enumerate(evs):
+                for e in ev:
+                    e.record(stream)          # create the handles before the library records them again
+                B.set_profile_events(ev)
                 step_eager(3 + i)
-            B.lib().base_profile_ffn_events(None, None)
+            B.set_profile_events(None)
         stream.synchronize()
-        # (in a stack every layer re-records the pair, so this is the last layer's FFN)
-        ffn_us = statistics.mean(a.elapsed_time(b) for a, b in evs) * 1e3
+        # (in a stack every layer re-records the events, so these are the last layer's kernels)
+        stage_us = {name: statistics.mean(ev[j].elapsed_time(ev[j + 1]) for ev in evs) * 1e3
+                    for j, name in enumerate(B.PROFILE_STAGES)}
+        ffn_us = stage_us["expert_ffn"]
 
     # ---- unlimited budget (dense batch-union step) for the speed-up, same protocol
     ms_dense = None
-    if not args.no_dense:
+    if not args.no_dense and not args.profile:
         with torch.cuda.stream(stream):
             for r in range(1 if stack else n_rep):
                 step_eager(r, cfg.E)
@@ -310,7 +312,7 @@ def run_ours(args, cfg, T, M):
 
     # ---- end to end through the host entry point (pinned host buffers, copies inside the timed region)
     e2e = None
-    if not stack:
+    if not stack and not args.profile:
         hws = B.alloc_workspace(B.layer_host_workspace_bytes(*shape, T), dev)
         h_in = [torch.from_numpy(wl.hidden_bits(cfg, T, layer=base_layer + r).view(np.int16)).view(torch.bfloat16).pin_memory()
                 for r in range(n_rep)]
@@ -371,8 +373,9 @@ def run_ours(args, cfg, T, M):
                             "peak": hbm_peak, "unit": "GB/s", "frac": ach / hbm_peak, "traffic": None,
                             "us_per_launch": ffn_us, "peak_kind": f"of {peak_kind}",
                             "algorithmic_bytes_per_launch": fb}
+        line["kernel_us"] = stage_us
     # CPU baseline: the oracle, as it stands, on this machine's host cores
-    if not args.no_cpu:
+    if not args.no_cpu and not args.profile:
         reps = 2 if cfg.expert_bytes < (64 << 20) else 1
         best, cores, _ = oracle_step_seconds(cfg if not stack else wl.CONFIGS["qwen3"], T, M, reps)
         scale = cfg.layers if stack else 1
@@ -395,6 +398,8 @@ def main():
     ap.add_argument("--batch", type=int, default=None)
     ap.add_argument("--no-cpu", action="store_true", help="skip the oracle timing")
     ap.add_argument("--no-dense", action="store_true", help="skip the unlimited-budget run")
+    ap.add_argument("--profile", action="store_true",
+                    help="only the warm-up and the timed steps (for a short run under a profiler)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     from paper_2609_36222_b200 import workloads as wl

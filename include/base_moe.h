@@ -179,12 +179,15 @@ int base_moe_decode_stack(const base_layer_shape* shape, const base_layer_weight
                           void* workspace, size_t workspace_bytes, void* stream);
 
 /*
- * Measurement hook (no counterpart in the paper). While a pair of cudaEvent_t handles is set for the
- * calling thread, every layer enqueued by that thread records `start_event` on the stream just before
- * its expert-FFN kernels and `stop_event` just after them, so a benchmark can time the dominant
- * kernels inside a full step. Pass NULL, NULL to switch it off. Not for use during stream capture.
+ * Measurement hook (no counterpart in the paper). While an array of BASE_PROFILE_EVENTS cudaEvent_t
+ * handles is set for the calling thread, every layer enqueued by that thread records them on its
+ * stream: [0] before the first kernel, [1] after the router/predictor GEMV, [2] after the routing
+ * kernel, [3] after the gather, [4] after the expert-FFN kernels, [5] after the combine. A benchmark
+ * can thus time each kernel inside a full step. The array is copied; pass NULL to switch the hook
+ * off. Not for use during stream capture.
  */
-int base_profile_ffn_events(void* start_event, void* stop_event);
+#define BASE_PROFILE_EVENTS 6
+int base_profile_events(void* const* events);
 
 /* Number of kernels the last successful base_moe_decode_layer call on this thread enqueued. */
 int base_last_launch_count(void);

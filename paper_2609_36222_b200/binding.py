@@ -24,7 +24,7 @@ DEV_NONFINITE_SCORE, DEV_WAIT_EXPIRED, DEV_BAD_INDEX = 1, 2, 4
 EXPORTS = (
     "base_predict_costs", "base_aggregate_select", "base_moe_decode_layer_workspace_bytes",
     "base_moe_decode_layer", "base_moe_decode_layer_host_workspace_bytes", "base_moe_decode_layer_host",
-    "base_moe_decode_stack_workspace_bytes", "base_moe_decode_stack", "base_profile_ffn_events",
+    "base_moe_decode_stack_workspace_bytes", "base_moe_decode_stack", "base_profile_events",
     "base_last_launch_count",
     "base_status_string", "base_last_cuda_error",
 )
@@ -79,7 +79,7 @@ def lib():
     L.base_moe_decode_stack_workspace_bytes.restype = C.c_size_t
     L.base_moe_decode_stack.argtypes = [C.POINTER(LayerShape), C.POINTER(LayerWeights), ip, vp, ip, ip, vp,
                                         C.POINTER(LayerOptions), vp, vp, C.c_size_t, vp]
-    L.base_profile_ffn_events.argtypes = [vp, vp]
+    L.base_profile_events.argtypes = [C.POINTER(C.c_void_p)]
     L.base_last_launch_count.restype = ip
     L.base_status_string.argtypes = [ip]
     L.base_status_string.restype = C.c_char_p
@@ -240,3 +240,16 @@ def base_moe_decode_stack(shape, weights_list, hidden, budget, out, workspace, n
 
 def last_launch_count():
     return lib().base_last_launch_count()
+
+
+PROFILE_STAGES = ("router_predictor_gemv", "routing", "gather", "expert_ffn", "combine")
+
+
+def set_profile_events(events):
+    """events: list of 6 torch.cuda.Event(enable_timing=True) already recorded once, or None to switch off."""
+    if events is None:
+        _check(lib().base_profile_events(None))
+        return
+    assert len(events) == 6
+    arr = (C.c_void_p * 6)(*[e.cuda_event for e in events])
+    _check(lib().base_profile_events(arr))

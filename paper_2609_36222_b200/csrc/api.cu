@@ -1,5 +1,6 @@
 // C-ABI entry points: argument checks, workspace carving, kernel sequencing. No device allocation,
 // no synchronisation (except the *_host entry point, which waits for its own copies).
+#include <stdlib.h>
 #include <string.h>
 
 #include "common.cuh"
@@ -11,7 +12,12 @@ namespace {
 
 thread_local int g_last_cuda_error = 0;
 thread_local int g_last_launches = 0;
-thread_local cudaEvent_t g_ev_start = nullptr, g_ev_stop = nullptr;
+thread_local cudaEvent_t g_ev[BASE_PROFILE_EVENTS] = {};
+thread_local bool g_ev_on = false;
+
+inline void mark(int i, cudaStream_t st) {
+  if (g_ev_on && g_ev[i]) cudaEventRecord(g_ev[i], st);
+}
 
 inline int cuda_fail(cudaError_t e) {
   g_last_cuda_error = int(e);
@@ -46,16 +52,22 @@ int enqueue_layer(const LayerCall& c, const Workspace& ws, cudaStream_t st, int*
   const base_layer_shape& s = *c.shape;
   cudaError_t e;
   const float* logits = c.router_logits;
-  e = launch_route_scores(c.hidden, c.w->router_w, c.w->router_bias, c.w->pred_A, c.w->pred_b,
-                          logits ? nullptr : ws.logits, ws.shat, c.T, s.d, s.E, st);
+  mark(0, st);
+  e = launch_route_scores(c.hidden, c.w->router_w, c.w->router_bias, c.w->pred_A, logits ? nullptr : ws.logits,
+                          ws.raw, ws.znorm2, c.T, s.d, s.E, st);
   if (e != cudaSuccess) return cuda_fail(e);
   ++*launches;
+  mark(1, st);
   if (!logits) logits = ws.logits;
 
   RoutingArgs ra{};
   ra.logits = logits;
-  ra.shat = ws.shat;
+  ra.raw = ws.raw;
+  ra.znorm2 = ws.znorm2;
+  ra.pred_b = c.w->pred_b;
   ra.forced_mask = c.forced_mask;
+  ra.hidden = static_cast<const __nv_bfloat16*>(c.hidden);
+  ra.d = s.d;
   ra.T = c.T;
   ra.E = s.E;
   ra.K = s.K;
@@ -66,24 +78,29 @@ int enqueue_layer(const LayerCall& c, const Workspace& ws, cudaStream_t st, int*
   ra.dbg = c.dbg;
   e = launch_routing(ra, st);
   if (e != cudaSuccess) return cuda_fail(e);
+#ifdef BASE_ROUTING_TIMING
+  if (getenv("BASE_DOUBLE_ROUTING")) launch_routing(ra, st);
+#endif
   ++*launches;
+  mark(2, st);
 
   e = launch_gather(c.hidden, ws, c.T, s.K, s.d, st);
   if (e != cudaSuccess) return cuda_fail(e);
   ++*launches;
 
-  if (g_ev_start) cudaEventRecord(g_ev_start, st);
+  mark(3, st);
   if (c.opt.ffn_impl == 1) {
     e = launch_ffn_simple(s, *c.w, ws, st, launches);
   } else {
     e = launch_ffn_tc(s, *c.w, ws, c.T, st, launches);
   }
   if (e != cudaSuccess) return cuda_fail(e);
-  if (g_ev_stop) cudaEventRecord(g_ev_stop, st);
+  mark(4, st);
 
   e = launch_combine(ws, c.hidden, c.out, c.opt.out_is_fp32, c.x_next, c.T, s.K, s.d, st);
   if (e != cudaSuccess) return cuda_fail(e);
   ++*launches;
+  mark(5, st);
   return BASE_OK;
 }
 
@@ -252,10 +269,9 @@ int base_moe_decode_stack(const base_layer_shape* shape, const base_layer_weight
   return BASE_OK;
 }
 
-int base_profile_ffn_events(void* start_event, void* stop_event) {
-  if ((start_event == nullptr) != (stop_event == nullptr)) return BASE_ERR_INVALID_ARG;
-  g_ev_start = static_cast<cudaEvent_t>(start_event);
-  g_ev_stop = static_cast<cudaEvent_t>(stop_event);
+int base_profile_events(void* const* events) {
+  g_ev_on = events != nullptr;
+  for (int i = 0; i < BASE_PROFILE_EVENTS; ++i) g_ev[i] = events ? static_cast<cudaEvent_t>(events[i]) : nullptr;
   return BASE_OK;
 }
 

@@ -46,7 +46,8 @@ __device__ __forceinline__ float silu_f(float x) { return x / (1.0f + expf(-x));
 // Pointers into the caller's workspace for one layer call (all device memory).
 struct Workspace {
   float* logits;          // [T,E]
-  float* shat;            // [T,E] predicted log-energy of every (token, expert) pair
+  float* raw;             // [T,E] a_e . z_t for every (token, expert) pair
+  float* znorm2;          // [T] ||z_t||^2
   float* costs;           // [T,E]
   int32_t* topk_ids;      // [T,K]
   float* topk_w;          // [T,K]
@@ -62,6 +63,8 @@ struct Workspace {
   int32_t* seg_expert;    // [max_segs] work segments: one expert, at most kSegTokens tokens
   int32_t* seg_offset;    // [max_segs] first sorted row of the segment
   int32_t* seg_count;     // [max_segs]
+  float* tok_m;           // [T] max logit of the token
+  float* tok_S;           // [T] softmax denominator over the original top-K
   int32_t* counters;      // [16 + E]: 0 n_dispatched, 1 n_segments, 2 status, 3 total slots, 4.. tickets; 16.. per-expert ready
   __nv_bfloat16* x_sorted; // [T*K + pad, d] token inputs in expert-sorted order
   __nv_bfloat16* h;        // [T*K + pad, I] silu(gate) * up, expert-sorted
@@ -95,7 +98,8 @@ inline Workspace carve_workspace(void* base_ptr, const base_layer_shape& s, int 
   w.ypair = static_cast<float*>(take(TK * s.d * 4, 1024));
   w.x_next = static_cast<__nv_bfloat16*>(take(size_t(T) * s.d * 2, 1024));
   w.logits = static_cast<float*>(take(TE * 4, 256));
-  w.shat = static_cast<float*>(take(TE * 4, 256));
+  w.raw = static_cast<float*>(take(TE * 4, 256));
+  w.znorm2 = static_cast<float*>(take(size_t(T) * 4, 256));
   w.costs = static_cast<float*>(take(TE * 4, 256));
   w.topk_ids = static_cast<int32_t*>(take(TK * 4, 256));
   w.topk_w = static_cast<float*>(take(TK * 4, 256));
@@ -111,6 +115,8 @@ inline Workspace carve_workspace(void* base_ptr, const base_layer_shape& s, int 
   w.seg_expert = static_cast<int32_t*>(take(size_t(segs) * 4, 256));
   w.seg_offset = static_cast<int32_t*>(take(size_t(segs) * 4, 256));
   w.seg_count = static_cast<int32_t*>(take(size_t(segs) * 4, 256));
+  w.tok_m = static_cast<float*>(take(size_t(T) * 4, 256));
+  w.tok_S = static_cast<float*>(take(size_t(T) * 4, 256));
   w.counters = static_cast<int32_t*>(take(size_t(kCtrReady + s.E) * 4, 256));
   w.bytes = align_up(off, 1024);
   return w;
@@ -120,9 +126,12 @@ inline Workspace carve_workspace(void* base_ptr, const base_layer_shape& s, int 
 
 struct RoutingArgs {
   const float* logits;        // [T,E] logits to route on
-  const float* shat;          // [T,E]
+  const float* raw;           // [T,E] a_e . z_t
+  const float* znorm2;        // [T]
+  const float* pred_b;        // [E]
   const uint8_t* forced_mask; // or nullptr
-  int T, E, K, M, gate_rule, fill_rule;
+  const __nv_bfloat16* hidden; // [T,d] token inputs (gathered into expert-sorted order)
+  int T, E, K, M, d, gate_rule, fill_rule;
   Workspace ws;
   base_layer_debug dbg;       // zero-initialised when the caller passed none
 };
@@ -132,8 +141,8 @@ cudaError_t launch_predict_costs(const void* hidden, const int32_t* ids, const f
 cudaError_t launch_aggregate_select(const float* costs, int T, int E, int M, float* scores, int32_t* sel,
                                     uint8_t* mask, cudaStream_t st);
 cudaError_t launch_route_scores(const void* hidden, const void* router_w, const float* router_bias,
-                                const void* pred_A, const float* pred_b, float* logits_out, float* shat,
-                                int T, int d, int E, cudaStream_t st);
+                                const void* pred_A, float* logits_out, float* raw, float* znorm2, int T, int d,
+                                int E, cudaStream_t st);
 cudaError_t launch_routing(const RoutingArgs& a, cudaStream_t st);
 cudaError_t launch_gather(const void* hidden, const Workspace& ws, int T, int K, int d, cudaStream_t st);
 cudaError_t launch_combine(const Workspace& ws, const void* hidden, void* out, int out_is_fp32, void* x_next,

@@ -1,15 +1,23 @@
 // Grouped SwiGLU expert FFN for sm_100a: TMA-staged weight streaming + tcgen05 MMA with TMEM
 // accumulators (Eq. moe_latency: the step is bound by fetching the dispatched experts' weights).
 //
-// Orientation ("swap-AB"): the weight rows are the MMA M axis (128 rows per tile, K-major, streamed
-// once, fully sequential in DRAM), the expert's tokens are the N axis (16..128 per work unit).
-//   gate/up pass: A = [64 rows of W_gate ; the same 64 rows of W_up] (two TMA boxes stacked in one
-//                 128-row tile), B = the expert's token inputs, D[0:64] = gate, D[64:128] = up;
+// Orientation ("swap-AB"): the weight rows are the MMA M axis (128 rows per tile, K-major, read
+// exactly once), the expert's tokens are the N axis (16..128 per work unit).
+//   gate/up pass: A = [64 rows of W_gate ; the same 64 rows of W_up] stacked in one 128-row tile,
+//                 B = the expert's token inputs, D[0:64] = gate, D[64:128] = up;
 //                 epilogue: h = silu(gate) * up -> bf16, expert-sorted rows.
 //   down pass:    A = 128 rows of W_down, B = the expert's h rows, D -> fp32 output per routed pair.
 // One persistent CTA per SM, warp-specialised: warp 0 issues TMA, warp 1 issues MMA and owns the
 // TMEM allocation, warps 2-5 drain the accumulators. Shared-memory stages and the two accumulator
 // stages are handed over with mbarriers, so the weight stream never waits for an epilogue.
+//
+// The single issuing threads are the scarce resource (a TMA or mbarrier instruction costs on the
+// order of a hundred cycles to issue), so a stage is made large and cheap to fill: it holds two
+// k-blocks (32 KB of weights) and is filled by ONE tensor-map box per operand. The weight box is
+// four-dimensional (64 elements, rows, {gate, up}, k-block) so that gate rows, up rows and both
+// k-blocks land in shared memory already in the layout the MMA descriptors expect; the token box
+// comes from a tensor map whose box height equals the padded token count of the unit.
+//
 // Every wait is bounded: on expiry the CTA raises an abort flag, all roles leave their loops, TMEM
 // is freed and BASE_DEV_WAIT_EXPIRED is OR-ed into the status word.
 #include <cuda.h>
@@ -23,41 +31,62 @@ namespace base {
 
 namespace {
 
-constexpr int kStages = 5;
 constexpr int kBlockK = 64;                 // bf16 per k-block = one 128-byte swizzled row
-constexpr int kTileABytes = 128 * 128;      // 128 rows x 128 B
-constexpr int kTileBBytes = kSegTokens * 128;
-constexpr int kStageBytes = kTileABytes + kTileBBytes;
-constexpr int kExBytes = kSegTokens * 64 * 4;  // up-projection exchange buffer [token][row] fp32
+constexpr int kKbPerStage = 2;              // k-blocks per pipeline stage
+constexpr int kTileABytes = 128 * 128;      // one k-block of the weight tile: 128 rows x 128 B
 constexpr int kThreads = 192;
-constexpr int kAccCols = kSegTokens;        // TMEM columns per accumulator stage
-constexpr int kTmemCols = 2 * kAccCols;
-constexpr int kBoxRowsB = 16;
-constexpr uint32_t kSpinLimit = 1u << 22;
-constexpr unsigned long long kWaitNs = 2000000000ull;  // 2 s
+constexpr int kMaxStages = 8;
+constexpr int kSmemLimit = 227 * 1024;      // dynamic shared memory one CTA may opt in to
+constexpr int kNumBMaps = kSegTokens / 16;  // token-tile tensor maps: box heights 16, 32, ..., 128
+constexpr uint32_t kSpinLimit = 1u << 26;
+constexpr long long kWaitCycles = 4000000000ll;   // about 2 s of SM clock
+
+// Shared-memory plan for work units of at most kMaxN tokens: the smaller the token tile, the more
+// weight stages fit.
+template <int kMaxN>
+struct Plan {
+  static constexpr int kTileBBytes = kMaxN * 128;                                  // per k-block
+  static constexpr int kStageBytes = kKbPerStage * (kTileABytes + kTileBBytes);
+  static constexpr int kExBytes = kMaxN * 64 * 4;   // up-projection exchange buffer [token][row] fp32
+  static constexpr int kFixed = 1024 /*alignment slack*/ + 512 /*barriers*/;
+  static constexpr int kFit = (kSmemLimit - kFixed - kExBytes) / kStageBytes;
+  static constexpr int kStages = kFit < kMaxStages ? kFit : kMaxStages;
+  static constexpr int kAccCols = kMaxN < 32 ? 32 : kMaxN;   // TMEM columns per accumulator stage
+  static constexpr int kTmemCols = 2 * kAccCols;
+  static constexpr size_t kSmemBytes = size_t(kFixed) + size_t(kStages) * kStageBytes + kExBytes;
+  static_assert(kStages >= 2, "need at least two stages");
+};
 
 struct Bars {
-  unsigned long long full[kStages];
-  unsigned long long empty[kStages];
+  unsigned long long full[kMaxStages];
+  unsigned long long empty[kMaxStages];
   unsigned long long acc_full[2];
   unsigned long long acc_empty[2];
   uint32_t tmem_base;
   int abort_flag;
 };
+static_assert(sizeof(Bars) <= 512, "barrier block must fit its reserved space");
 
-constexpr size_t kSmemBytes = 1024 + size_t(kStages) * kStageBytes + kExBytes + sizeof(Bars) + 64;
+// Tensor maps of one pass. a: weights; a2: second weight matrix when gate and up cannot share one
+// map; b[i]: token operand with a box of 16*(i+1) rows.
+struct MapSet {
+  CUtensorMap a;
+  CUtensorMap a2;
+  CUtensorMap b[kNumBMaps];
+};
 
 struct FfnParams {
   const int32_t* seg_expert;
   const int32_t* seg_offset;
   const int32_t* seg_count;
   int32_t* counters;
-  __nv_bfloat16* h;   // gate/up pass output
-  float* ypair;       // down pass output
-  int rows_per_expert;  // I (gate/up) or d (down): rows of one expert in the A tensor map
+  __nv_bfloat16* h;     // gate/up pass output
+  float* ypair;         // down pass output
+  int rows_per_expert;  // I (gate/up) or d (down): rows of one expert in the weight tensor map
   int tiles;            // work units per segment
   int kblocks;          // K extent / 64
   int I, d;
+  int split_a;          // gate/up pass: 1 = gate and up come from two maps (two boxes per k-block)
 };
 
 // ------------------------------------------------------------------------------------------- PTX wrappers
@@ -83,21 +112,19 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-__device__ __forceinline__ unsigned long long global_ns() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-  return t;
-}
 // Bounded wait. Returns false when the wait ran out or another role has raised the abort flag.
-__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+// A failed try_wait already suspends the thread for a hardware-defined interval; `sleep_ns` adds a
+// back-off for roles whose waits are long (the epilogue), so that they do not load the barrier unit.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t sleep_ns = 0) {
   if (mbar_try_wait(bar, parity)) return true;
-  const unsigned long long t0 = global_ns();
+  const long long t0 = clock64();
+#pragma unroll 1
   for (uint32_t it = 0; it < kSpinLimit; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
-    if ((it & 63u) == 63u) {
+    if (sleep_ns) __nanosleep(sleep_ns);
+    if ((it & 255u) == 255u) {
       if (*abort_flag) return false;
-      if (global_ns() - t0 > kWaitNs) break;
-      __nanosleep(64);
+      if (clock64() - t0 > kWaitCycles) break;
     }
   }
   if (mbar_try_wait(bar, parity)) return true;
@@ -105,10 +132,17 @@ __device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile i
   return false;
 }
 
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar) {
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, int c0, int c1, int c2, uint32_t bar) {
   asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
-      "l"(tm), "r"(x), "r"(y), "r"(bar)
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(dst),
+      "l"(tm), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* tm, int c0, int c1, int c2, int c3, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];" ::"r"(
+          dst),
+      "l"(tm), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar)
       : "memory");
 }
 
@@ -193,19 +227,21 @@ __device__ __forceinline__ Unit decode_unit(const FfnParams& p, int u) {
 }
 
 // ------------------------------------------------------------------------------------------- the kernel
-template <int kPhase>
-__global__ void __launch_bounds__(kThreads, 1)
-ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_a0, const __grid_constant__ CUtensorMap tm_a1,
-              const __grid_constant__ CUtensorMap tm_b, const FfnParams p) {
+template <int kPhase, int kMaxN>
+__global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_constant__ MapSet maps, const FfnParams p) {
+  using P = Plan<kMaxN>;
+  constexpr int kStages = P::kStages, kStageBytes = P::kStageBytes, kAccCols = P::kAccCols, kTmemCols = P::kTmemCols;
+  constexpr int kStageABytes = kKbPerStage * kTileABytes;
   extern __shared__ unsigned char smem_raw[];
   unsigned char* base_ptr = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   unsigned char* stages = base_ptr;
   float* ex = reinterpret_cast<float*>(base_ptr + size_t(kStages) * kStageBytes);
-  Bars* bars = reinterpret_cast<Bars*>(base_ptr + size_t(kStages) * kStageBytes + kExBytes);
+  Bars* bars = reinterpret_cast<Bars*>(base_ptr + size_t(kStages) * kStageBytes + P::kExBytes);
   volatile int* abort_flag = &bars->abort_flag;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_units = p.counters[kCtrSegments] * p.tiles;
+  const int n_steps = (p.kblocks + kKbPerStage - 1) / kKbPerStage;   // pipeline stages per unit
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
@@ -218,9 +254,8 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_a0, const __grid_constant__
     }
     bars->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_a0) : "memory");
-    asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_b) : "memory");
-    if (kPhase == 1) asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_a1) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&maps.a) : "memory");
+    if (kPhase == 1 && p.split_a) asm volatile("prefetch.tensormap [%0];" ::"l"(&maps.a2) : "memory");
   }
   if (warp == 1) tmem_alloc(smem_u32(&bars->tmem_base), kTmemCols);
   tcgen05_fence_before();
@@ -237,22 +272,34 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_a0, const __grid_constant__
       for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
         const Unit un = decode_unit(p, u);
         const int arow = un.expert * p.rows_per_expert + un.tile * (kPhase == 1 ? 64 : 128);
-        for (int kb = 0; kb < p.kblocks; ++kb) {
+        const CUtensorMap* tm_b = &maps.b[(un.npad >> 4) - 1];
+        const uint32_t bytes = uint32_t(kKbPerStage * (kTileABytes + un.npad * 128));
+        for (int st = 0; st < n_steps; ++st) {
           if (!mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1u, abort_flag)) {
             ok = false;
             break;
           }
+          const int kb = st * kKbPerStage;
           const uint32_t full = smem_u32(&bars->full[stage]);
           const uint32_t sa = smem_u32(stages + size_t(stage) * kStageBytes);
-          const uint32_t sb = sa + kTileABytes;
-          mbar_expect_tx(full, uint32_t(kTileABytes + un.npad * 128));
+          const uint32_t sb = sa + kStageABytes;
+          // k-blocks past the end of K are out of the tensor's bounds and arrive as zeros; the box
+          // always delivers its full byte count.
+          mbar_expect_tx(full, bytes);
           if (kPhase == 1) {
-            tma_load_2d(sa, &tm_a0, kb * kBlockK, arow, full);
-            tma_load_2d(sa + kTileABytes / 2, &tm_a1, kb * kBlockK, arow, full);
+            if (!p.split_a) {
+              tma_load_4d(sa, &maps.a, 0, arow, 0, kb, full);      // {elem, row, gate|up, k-block}
+            } else {
+#pragma unroll
+              for (int j = 0; j < kKbPerStage; ++j) {
+                tma_load_3d(sa + j * kTileABytes, &maps.a, 0, arow, kb + j, full);
+                tma_load_3d(sa + j * kTileABytes + kTileABytes / 2, &maps.a2, 0, arow, kb + j, full);
+              }
+            }
           } else {
-            tma_load_2d(sa, &tm_a0, kb * kBlockK, arow, full);
+            tma_load_3d(sa, &maps.a, 0, arow, kb, full);             // {elem, row, k-block}
           }
-          for (int j = 0; j < un.npad; j += kBoxRowsB) tma_load_2d(sb + j * 128, &tm_b, kb * kBlockK, un.offset + j, full);
+          tma_load_3d(sb, tm_b, 0, un.offset, kb, full);
           if (++stage == kStages) {
             stage = 0;
             phase ^= 1u;
@@ -273,18 +320,25 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_a0, const __grid_constant__
         tcgen05_fence_after();
         const uint32_t d_tmem = tmem_base + uint32_t(acc * kAccCols);
         const uint32_t idesc = make_idesc(un.npad);
-        for (int kb = 0; kb < p.kblocks; ++kb) {
+        const uint32_t tile_b = uint32_t(un.npad * 128);
+        for (int st = 0; st < n_steps; ++st) {
           if (!mbar_wait(smem_u32(&bars->full[stage]), phase, abort_flag)) {
             ok = false;
             break;
           }
           tcgen05_fence_after();
           const uint32_t sa = smem_u32(stages + size_t(stage) * kStageBytes);
-          const uint64_t adesc = make_smem_desc(sa);
-          const uint64_t bdesc = make_smem_desc(sa + kTileABytes);
+          const uint32_t sb = sa + kStageABytes;
 #pragma unroll
-          for (int k4 = 0; k4 < kBlockK / 16; ++k4)
-            umma_bf16(d_tmem, adesc + uint64_t(k4 * 2), bdesc + uint64_t(k4 * 2), idesc, uint32_t((kb | k4) != 0));
+          for (int j = 0; j < kKbPerStage; ++j) {
+            if (st * kKbPerStage + j < p.kblocks) {
+              const uint64_t adesc = make_smem_desc(sa + j * kTileABytes);
+              const uint64_t bdesc = make_smem_desc(sb + j * tile_b);
+#pragma unroll
+              for (int k4 = 0; k4 < kBlockK / 16; ++k4)
+                umma_bf16(d_tmem, adesc + uint64_t(k4 * 2), bdesc + uint64_t(k4 * 2), idesc, uint32_t((st | j | k4) != 0));
+            }
+          }
           umma_commit(smem_u32(&bars->empty[stage]));
           if (++stage == kStages) {
             stage = 0;
@@ -305,8 +359,10 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_a0, const __grid_constant__
     uint32_t acc_phase = 0;
     for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
       const Unit un = decode_unit(p, u);
-      const bool got = mbar_wait(smem_u32(&bars->acc_full[acc]), acc_phase, abort_flag);
-      if (!named_and(1, 128, got)) break;
+      int got = 0;
+      if (lane == 0) got = mbar_wait(smem_u32(&bars->acc_full[acc]), acc_phase, abort_flag, 128) ? 1 : 0;
+      got = __shfl_sync(0xffffffffu, got, 0);
+      if (!named_and(1, 128, got != 0)) break;
       tcgen05_fence_after();
       const uint32_t taddr = tmem_base + (uint32_t(q * 32) << 16) + uint32_t(acc * kAccCols);
       if (kPhase == 1) {
@@ -384,28 +440,41 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
+// A bf16 tensor map of rank <= 4 with 128-byte swizzle. dims/box are in elements (innermost first),
+// strides in bytes for dimensions 1.. (the innermost is contiguous).
 struct MapKey {
   const void* ptr;
-  uint64_t rows, cols;
-  uint32_t box_rows;
-  bool operator==(const MapKey& o) const { return ptr == o.ptr && rows == o.rows && cols == o.cols && box_rows == o.box_rows; }
+  uint32_t rank;
+  uint64_t dims[4];
+  uint64_t strides[3];
+  uint32_t box[4];
+  bool operator==(const MapKey& o) const {
+    if (ptr != o.ptr || rank != o.rank) return false;
+    for (int i = 0; i < 4; ++i)
+      if (dims[i] != o.dims[i] || box[i] != o.box[i]) return false;
+    for (int i = 0; i < 3; ++i)
+      if (strides[i] != o.strides[i]) return false;
+    return true;
+  }
 };
 struct MapKeyHash {
   size_t operator()(const MapKey& k) const {
-    size_t h = reinterpret_cast<size_t>(k.ptr);
-    h ^= k.rows * 0x9E3779B97F4A7C15ull + (h << 6) + (h >> 2);
-    h ^= k.cols * 0xBF58476D1CE4E5B9ull + (h << 6) + (h >> 2);
-    h ^= k.box_rows * 0x94D049BB133111EBull + (h << 6) + (h >> 2);
-    return h;
+    uint64_t h = reinterpret_cast<uint64_t>(k.ptr) * 0x9E3779B97F4A7C15ull + k.rank;
+    for (int i = 0; i < 4; ++i) h = (h ^ (k.dims[i] + k.box[i] * 0x10001ull)) * 0xBF58476D1CE4E5B9ull;
+    for (int i = 0; i < 3; ++i) h = (h ^ k.strides[i]) * 0x94D049BB133111EBull;
+    return size_t(h ^ (h >> 29));
   }
 };
 
-// 2-D bf16 tensor [rows, cols] (cols contiguous), box = [box_rows, 64 cols], 128-byte swizzle. Cached: the
-// encoding is a pure function of the key.
-bool tensor_map_2d(const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows, CUtensorMap* out) {
+// Cached: the encoding is a pure function of the key.
+bool encode_map(MapKey key, CUtensorMap* out) {
   static std::mutex mu;
   static std::unordered_map<MapKey, CUtensorMap, MapKeyHash> cache;
-  const MapKey key{ptr, rows, cols, box_rows};
+  for (uint32_t i = key.rank; i < 4; ++i) {
+    key.dims[i] = 1;
+    key.box[i] = 1;
+  }
+  for (uint32_t i = key.rank > 0 ? key.rank - 1 : 0; i < 3; ++i) key.strides[i] = 0;
   {
     std::lock_guard<std::mutex> g(mu);
     auto it = cache.find(key);
@@ -416,22 +485,67 @@ bool tensor_map_2d(const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_r
   }
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
-  const cuuint64_t dims[2] = {cols, rows};
-  const cuuint64_t strides[1] = {cols * 2};
-  const cuuint32_t box[2] = {uint32_t(kBlockK), box_rows};
-  const cuuint32_t estr[2] = {1, 1};
+  cuuint64_t dims[4], strides[3];
+  cuuint32_t box[4], estr[4] = {1, 1, 1, 1};
+  for (int i = 0; i < 4; ++i) {
+    dims[i] = key.dims[i];
+    box[i] = key.box[i];
+  }
+  for (int i = 0; i < 3; ++i) strides[i] = key.strides[i];
   CUtensorMap m;
-  CUresult r = fn(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+  CUresult r = fn(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, key.rank, const_cast<void*>(key.ptr), dims, strides, box, estr,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return false;
   {
     std::lock_guard<std::mutex> g(mu);
-    if (cache.size() > 4096) cache.clear();
+    if (cache.size() > 8192) cache.clear();
     cache.emplace(key, m);
   }
   *out = m;
   return true;
+}
+
+// [rows, cols] row-major matrix seen as {64 elements, rows, k-blocks}: coordinate 2 steps 128 bytes
+// along a row, so a box {64, box_rows, n_kb} lands as consecutive k-block tiles.
+bool map_rows_kblocks(const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows, uint32_t box_kb, CUtensorMap* out) {
+  MapKey k{};
+  k.ptr = ptr;
+  k.rank = 3;
+  k.dims[0] = kBlockK;
+  k.dims[1] = rows;
+  k.dims[2] = cols / kBlockK;
+  k.strides[0] = cols * 2;
+  k.strides[1] = kBlockK * 2;
+  k.box[0] = kBlockK;
+  k.box[1] = box_rows;
+  k.box[2] = box_kb;
+  return encode_map(k, out);
+}
+
+// Gate and up matrices seen through one map {64 elements, rows, {gate, up}, k-blocks}: the third
+// coordinate steps from W_gate to W_up, which works whenever W_up lies above W_gate at a distance
+// the tensor map can express.
+bool map_gate_up(const void* gate, const void* up, uint64_t rows, uint64_t cols, CUtensorMap* out) {
+  const uintptr_t g = reinterpret_cast<uintptr_t>(gate), u = reinterpret_cast<uintptr_t>(up);
+  if (u <= g) return false;
+  const uint64_t delta = u - g;
+  if ((delta & 15u) != 0 || delta >= (1ull << 40)) return false;
+  MapKey k{};
+  k.ptr = gate;
+  k.rank = 4;
+  k.dims[0] = kBlockK;
+  k.dims[1] = rows;
+  k.dims[2] = 2;
+  k.dims[3] = cols / kBlockK;
+  k.strides[0] = cols * 2;
+  k.strides[1] = delta;
+  k.strides[2] = kBlockK * 2;
+  k.box[0] = kBlockK;
+  k.box[1] = 64;
+  k.box[2] = 2;
+  k.box[3] = kKbPerStage;
+  return encode_map(k, out);
 }
 
 int sm_count() {
@@ -444,10 +558,34 @@ int sm_count() {
   return n;
 }
 
-template <int kPhase>
+template <int kPhase, int kMaxN>
 cudaError_t configure() {
-  static cudaError_t st = cudaFuncSetAttribute(ffn_tc_kernel<kPhase>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kSmemBytes));
+  static cudaError_t st = cudaFuncSetAttribute(ffn_tc_kernel<kPhase, kMaxN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                               int(Plan<kMaxN>::kSmemBytes));
   return st;
+}
+
+template <int kMaxN>
+cudaError_t launch_both(const MapSet& m1, const MapSet& m2, FfnParams p, const base_layer_shape& s, int segs,
+                        cudaStream_t st) {
+  cudaError_t e = configure<1, kMaxN>();
+  if (e != cudaSuccess) return e;
+  e = configure<2, kMaxN>();
+  if (e != cudaSuccess) return e;
+  p.rows_per_expert = s.I;
+  p.tiles = s.I / 64;
+  p.kblocks = s.d / kBlockK;
+  int grid = min(sm_count(), segs * p.tiles);
+  ffn_tc_kernel<1, kMaxN><<<grid, kThreads, Plan<kMaxN>::kSmemBytes, st>>>(m1, p);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  p.rows_per_expert = s.d;
+  p.tiles = s.d / 128;
+  p.kblocks = s.I / kBlockK;
+  p.split_a = 0;
+  grid = min(sm_count(), segs * p.tiles);
+  ffn_tc_kernel<2, kMaxN><<<grid, kThreads, Plan<kMaxN>::kSmemBytes, st>>>(m2, p);
+  return cudaGetLastError();
 }
 
 }  // namespace
@@ -455,20 +593,24 @@ cudaError_t configure() {
 cudaError_t launch_ffn_tc(const base_layer_shape& s, const base_layer_weights& w, const Workspace& ws, int T,
                           cudaStream_t st, int* launches) {
   const uint64_t slots = uint64_t(T) * s.K + kRowPad;
-  CUtensorMap tm_g, tm_u, tm_x, tm_d, tm_h;
-  if (!tensor_map_2d(w.w_gate, uint64_t(s.E) * s.I, s.d, 64, &tm_g) ||
-      !tensor_map_2d(w.w_up, uint64_t(s.E) * s.I, s.d, 64, &tm_u) ||
-      !tensor_map_2d(ws.x_sorted, slots, s.d, kBoxRowsB, &tm_x) ||
-      !tensor_map_2d(w.w_down, uint64_t(s.E) * s.d, s.I, 128, &tm_d) ||
-      !tensor_map_2d(ws.h, slots, s.I, kBoxRowsB, &tm_h))
-    return cudaErrorInvalidValue;
-  cudaError_t e = configure<1>();
-  if (e != cudaSuccess) return e;
-  e = configure<2>();
-  if (e != cudaSuccess) return e;
+  const uint64_t wrows = uint64_t(s.E) * s.I;
+  MapSet m1{}, m2{};
+  FfnParams p{};
+  if (map_gate_up(w.w_gate, w.w_up, wrows, s.d, &m1.a)) {
+    p.split_a = 0;
+  } else {
+    p.split_a = 1;
+    if (!map_rows_kblocks(w.w_gate, wrows, s.d, 64, 1, &m1.a) || !map_rows_kblocks(w.w_up, wrows, s.d, 64, 1, &m1.a2))
+      return cudaErrorInvalidValue;
+  }
+  if (!map_rows_kblocks(w.w_down, uint64_t(s.E) * s.d, s.I, 128, kKbPerStage, &m2.a)) return cudaErrorInvalidValue;
+  for (int i = 0; i < kNumBMaps; ++i) {
+    if (!map_rows_kblocks(ws.x_sorted, slots, s.d, 16 * (i + 1), kKbPerStage, &m1.b[i]) ||
+        !map_rows_kblocks(ws.h, slots, s.I, 16 * (i + 1), kKbPerStage, &m2.b[i]))
+      return cudaErrorInvalidValue;
+  }
 
   const int segs = max_segments(s.E, T, s.K);
-  FfnParams p{};
   p.seg_expert = ws.seg_expert;
   p.seg_offset = ws.seg_offset;
   p.seg_count = ws.seg_count;
@@ -477,22 +619,13 @@ cudaError_t launch_ffn_tc(const base_layer_shape& s, const base_layer_weights& w
   p.ypair = ws.ypair;
   p.I = s.I;
   p.d = s.d;
-
-  p.rows_per_expert = s.I;
-  p.tiles = s.I / 64;
-  p.kblocks = s.d / kBlockK;
-  int grid = min(sm_count(), segs * p.tiles);
-  ffn_tc_kernel<1><<<grid, kThreads, kSmemBytes, st>>>(tm_g, tm_u, tm_x, p);
-  e = cudaGetLastError();
-  if (e != cudaSuccess) return e;
-
-  p.rows_per_expert = s.d;
-  p.tiles = s.d / 128;
-  p.kblocks = s.I / kBlockK;
-  grid = min(sm_count(), segs * p.tiles);
-  ffn_tc_kernel<2><<<grid, kThreads, kSmemBytes, st>>>(tm_d, tm_d, tm_h, p);
+  // No expert can receive more tokens than the batch holds, which bounds the token tile.
+  cudaError_t e;
+  if (T <= 32) e = launch_both<32>(m1, m2, p, s, segs, st);
+  else if (T <= 64) e = launch_both<64>(m1, m2, p, s, segs, st);
+  else e = launch_both<128>(m1, m2, p, s, segs, st);
   *launches += 2;
-  return cudaGetLastError();
+  return e;
 }
 
 }  // namespace base

@@ -1,7 +1,6 @@
 // Routing side of the decode layer: router/predictor GEMV, predicted removal costs, batch
-// aggregation, top-M selection, restricted routing with backfill, and the expert-sorted
-// dispatch lists. Everything between the GEMV and the expert FFN runs in one CTA with no host
-// round trip.
+// aggregation, top-M selection, restricted routing with backfill, the expert-sorted dispatch
+// lists, the gather into expert order and the final combine. No step needs the host.
 #include <limits.h>
 #include <math.h>
 
@@ -121,336 +120,485 @@ cudaError_t launch_aggregate_select(const float* costs, int T, int E, int M, flo
 }
 
 // ------------------------------------------------------------------------------------------------
-// Router + predictor GEMV for every (token, expert) pair: logits[t,e] = z_t . W_r[e] + bias[e] and
-// shat[t,e] = a_e . z_t / ||z_t|| + b_e. grid = (E, token chunks); the two weight rows sit in shared
-// memory, each warp streams its tokens with 128-bit loads. Computing shat for all pairs (not only
-// the routed ones) removes the dependency on the top-K result; it costs one more 2*E*d-byte read.
+// Router + predictor GEMV for every (token, expert) pair on the warp-level tensor-core path:
+//   logits[t,e] = z_t . W_r[e] + bias[e]      raw[t,e] = z_t . a_e      znorm2[t] = ||z_t||^2
+// (the routing kernel turns raw into the predicted log-energy a_e . z_t/||z_t|| + b_e).
+// The 2E weight rows [W_r ; A] are the M axis (16 per CTA), 8 tokens the N axis, and the four warps
+// of a CTA split K. Each lane reads 16-byte pieces of its row and of its token directly in fragment
+// position: a dot product does not care about the order of k, so the same permutation of k is
+// applied to both operands and no shared-memory staging is needed. Computing raw for all pairs (not
+// only the routed ones) removes the dependency on the top-K result.
 // ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) route_scores_kernel(const __nv_bfloat16* __restrict__ hidden,
-                                                           const __nv_bfloat16* __restrict__ router_w,
-                                                           const float* __restrict__ router_bias,
-                                                           const __nv_bfloat16* __restrict__ pred_A,
-                                                           const float* __restrict__ pred_b,
-                                                           float* __restrict__ logits, float* __restrict__ shat,
-                                                           int T, int d, int E, int tokens_per_cta) {
-  extern __shared__ uint4 s_rows[];  // [2][d/8]
-  const int e = blockIdx.x;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
-  const int dv = d >> 3;
-  const bool do_logits = logits != nullptr;
-  for (int j = threadIdx.x; j < dv; j += blockDim.x) {
-    s_rows[j] = do_logits ? ldg16(router_w + size_t(e) * d + j * 8) : make_uint4(0, 0, 0, 0);
-    s_rows[dv + j] = ldg16(pred_A + size_t(e) * d + j * 8);
-  }
-  __syncthreads();
-  const int t0 = blockIdx.y * tokens_per_cta;
-  const int t1 = min(T, t0 + tokens_per_cta);
-  for (int t = t0 + warp; t < t1; t += nwarp) {
-    const __nv_bfloat16* z = hidden + size_t(t) * d;
-    float accL = 0.f, accA = 0.f, accZ = 0.f;
-    for (int j = lane; j < dv; j += 32) {
-      float fz[8], fr[8], fa[8];
-      unpack8(ldg16(z + j * 8), fz);
-      unpack8(s_rows[j], fr);
-      unpack8(s_rows[dv + j], fa);
+constexpr int kGemvWarps = 4;
+constexpr int kGemvBatch = 8;   // k32-blocks whose loads are in flight together
+
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                               uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ float sumsq_bf16x2(uint32_t w) {
+  const float lo = __uint_as_float(w << 16), hi = __uint_as_float(w & 0xffff0000u);
+  return lo * lo + hi * hi;
+}
+
+__global__ void __launch_bounds__(kGemvWarps * 32) route_scores_kernel(const __nv_bfloat16* __restrict__ hidden,
+                                                                       const __nv_bfloat16* __restrict__ router_w,
+                                                                       const float* __restrict__ router_bias,
+                                                                       const __nv_bfloat16* __restrict__ pred_A,
+                                                                       float* __restrict__ logits,
+                                                                       float* __restrict__ raw,
+                                                                       float* __restrict__ znorm2, int T, int d,
+                                                                       int E) {
+  __shared__ float s_part[kGemvWarps][16 * 8 + 8];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = lane >> 2, q = lane & 3;
+  const int r0 = blockIdx.x * 16, n0 = blockIdx.y * 8;
+  auto row_ptr = [&](int r) -> const __nv_bfloat16* {
+    r = min(r, 2 * E - 1);
+    if (r < E) return (router_w ? router_w : pred_A) + size_t(r) * d;   // router rows unused when logits are given
+    return pred_A + size_t(r - E) * d;
+  };
+  const __nv_bfloat16* pa = row_ptr(r0 + g);
+  const __nv_bfloat16* pb = row_ptr(r0 + g + 8);
+  const __nv_bfloat16* pz = hidden + size_t(min(n0 + g, T - 1)) * d;
+  const int nblk = d >> 5;
+  const int b_lo = (nblk * warp) / kGemvWarps, b_hi = (nblk * (warp + 1)) / kGemvWarps;
+  float c[4] = {0.f, 0.f, 0.f, 0.f};
+  float zz = 0.f;
+  for (int b0 = b_lo; b0 < b_hi; b0 += kGemvBatch) {
+    uint4 x[kGemvBatch], y[kGemvBatch], z[kGemvBatch];
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        accL = fmaf(fz[i], fr[i], accL);
-        accA = fmaf(fz[i], fa[i], accA);
-        accZ = fmaf(fz[i], fz[i], accZ);
+    for (int i = 0; i < kGemvBatch; ++i) {
+      if (b0 + i < b_hi) {
+        const int k = (b0 + i) * 32 + q * 8;
+        x[i] = ldg16(pa + k);
+        y[i] = ldg16(pb + k);
+        z[i] = ldg16(pz + k);
       }
     }
-    accL = warp_sum(accL);
-    accA = warp_sum(accA);
-    accZ = warp_sum(accZ);
-    if (lane == 0) {
-      if (do_logits) logits[size_t(t) * E + e] = accL + (router_bias ? router_bias[e] : 0.f);
-      shat[size_t(t) * E + e] = accA / fmaxf(sqrtf(accZ), 1e-30f) + pred_b[e];
+#pragma unroll
+    for (int i = 0; i < kGemvBatch; ++i) {
+      if (b0 + i < b_hi) {
+        mma_bf16_16816(c, x[i].x, y[i].x, x[i].y, y[i].y, z[i].x, z[i].y);
+        mma_bf16_16816(c, x[i].z, y[i].z, x[i].w, y[i].w, z[i].z, z[i].w);
+        zz += sumsq_bf16x2(z[i].x) + sumsq_bf16x2(z[i].y) + sumsq_bf16x2(z[i].z) + sumsq_bf16x2(z[i].w);
+      }
+    }
+  }
+  zz += __shfl_xor_sync(0xffffffffu, zz, 1);
+  zz += __shfl_xor_sync(0xffffffffu, zz, 2);
+  // c[0],c[1]: row g, tokens 2q, 2q+1; c[2],c[3]: row g+8, same tokens
+  s_part[warp][g * 8 + 2 * q] = c[0];
+  s_part[warp][g * 8 + 2 * q + 1] = c[1];
+  s_part[warp][(g + 8) * 8 + 2 * q] = c[2];
+  s_part[warp][(g + 8) * 8 + 2 * q + 1] = c[3];
+  if (q == 0) s_part[warp][128 + g] = zz;
+  __syncthreads();
+  {
+    const int i = threadIdx.x;   // 128 threads: one output each
+    float v = 0.f;
+#pragma unroll
+    for (int w = 0; w < kGemvWarps; ++w) v += s_part[w][i];
+    const int r = r0 + (i >> 3), t = n0 + (i & 7);
+    if (t < T && r < 2 * E) {
+      if (r < E) {
+        if (logits) logits[size_t(t) * E + r] = v + (router_bias ? router_bias[r] : 0.f);
+      } else {
+        raw[size_t(t) * E + (r - E)] = v;
+      }
+    }
+    if (blockIdx.x == 0 && i < 8 && n0 + i < T) {
+      float n2 = 0.f;
+#pragma unroll
+      for (int w = 0; w < kGemvWarps; ++w) n2 += s_part[w][128 + i];
+      znorm2[n0 + i] = n2;
     }
   }
 }
 
 cudaError_t launch_route_scores(const void* hidden, const void* router_w, const float* router_bias,
-                                const void* pred_A, const float* pred_b, float* logits_out, float* shat,
-                                int T, int d, int E, cudaStream_t st) {
-  int chunks = (2 * 148 + E - 1) / E;               // aim at >= 2 CTAs per SM
-  chunks = max(1, min(chunks, (T + 7) / 8));        // at least one token per warp
-  const int tpc = (T + chunks - 1) / chunks;
-  dim3 grid(E, (T + tpc - 1) / tpc);
-  route_scores_kernel<<<grid, 256, size_t(d) * 4, st>>>(
+                                const void* pred_A, float* logits_out, float* raw, float* znorm2, int T, int d,
+                                int E, cudaStream_t st) {
+  dim3 grid((2 * E + 15) / 16, (T + 7) / 8);
+  route_scores_kernel<<<grid, kGemvWarps * 32, 0, st>>>(
       static_cast<const __nv_bfloat16*>(hidden), static_cast<const __nv_bfloat16*>(router_w), router_bias,
-      static_cast<const __nv_bfloat16*>(pred_A), pred_b, logits_out, shat, T, d, E, tpc);
+      static_cast<const __nv_bfloat16*>(pred_A), logits_out, raw, znorm2, T, d, E);
   return cudaGetLastError();
 }
 
 // ------------------------------------------------------------------------------------------------
-// The routing kernel: one CTA.
-//   A  per token: top-K of the logits (value desc, id asc), q = exp(l - max), S = sum over R_t,
-//      w = q/S, predicted cost c = w^2 exp(shat)                                (Sec. 3.1, 3.4)
-//   B  D[u] = sum_t c[t,u]                                                      (Sec. 3.4)
-//   C  active set = top-M of D by rank counting                                 (Sec. 3.5)
-//   D  per token: K highest-ranked experts inside the active set, gate = q / S  (Sec. 3.5)
-//   E  expert-sorted dispatch: counts, offsets, row of every executed pair, work segments
+// The routing kernel: one thread-block cluster of kClusterCtas CTAs (hardware cluster barriers, all
+// CTAs co-scheduled, so no wait can starve). Stages:
+//   1  per token (one warp each): top-K of the logits (value desc, id asc), q = exp(l - max),
+//      S = sum over R_t, w = q/S, predicted cost c = w^2 exp(shat)                  (Sec. 3.1, 3.4)
+//   -- cluster barrier --
+//   2  every CTA: D[u] = sum_t c[t,u] in a fixed order                              (Sec. 3.4)
+//   3  every CTA: top-M of D by rank counting -> its own copy of the active mask    (Sec. 3.5)
+//      per token: K highest-ranked experts inside the active set, gate = q / S      (Sec. 3.5)
+//   -- cluster barrier --
+//   4  every CTA: tokens dispatched to each expert in token order, offsets by a scan of the counts,
+//      the row of every routed pair in the expert-sorted buffers.
+// Work that needs all tokens (2, 3a, 4) is repeated by every CTA instead of being shared, which
+// leaves two cluster barriers in the whole kernel. Everything is written for short dependent
+// chains: loads are issued in batches, the arg-max is two warp reductions, loop bounds that the
+// compiler must unroll are compile-time constants.
 // ------------------------------------------------------------------------------------------------
 constexpr int kNone = INT_MAX;
+constexpr int kClusterCtas = 8;
+constexpr int kRoutingThreads = 512;
+constexpr int kRoutingWarps = kRoutingThreads / 32;
 
-__device__ __forceinline__ void warp_argbest(float& v, int& idx) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    const float ov = __shfl_xor_sync(0xffffffffu, v, o);
-    const int oi = __shfl_xor_sync(0xffffffffu, idx, o);
-    if (oi != kNone && (idx == kNone || ov > v || (ov == v && oi < idx))) {
-      v = ov;
-      idx = oi;
-    }
-  }
+// Order-preserving map float -> uint32 (larger float <=> larger key). Key 0 is never produced by a
+// finite value or an infinity, so it stands for "no candidate".
+__device__ __forceinline__ uint32_t float_key(float f) {
+  const uint32_t b = __float_as_uint(f);
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+__device__ __forceinline__ float key_float(uint32_t k) {
+  return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
 }
 
-// Pick the best available entry of this warp's logit row and mark it taken. All lanes return it.
-__device__ __forceinline__ void take_best(const float (&v)[kMaxVals], uint32_t& avail, int lane, float& bv, int& bi) {
-  bv = -INFINITY;
-  bi = kNone;
+// Pick the best available entry of this warp's row (value desc, id asc) with two warp reductions and
+// mark it taken. Every lane returns the same (key, id); id == kNone when nothing is left.
+template <int NV>
+__device__ __forceinline__ void take_best(const uint32_t (&key)[NV], uint32_t& avail, int lane, uint32_t& gk, int& gi) {
+  uint32_t bk = 0;
+  int bi = kNone;
 #pragma unroll
-  for (int i = 0; i < kMaxVals; ++i) {
-    if ((avail >> i) & 1u) {
-      if (bi == kNone || v[i] > bv) {
-        bv = v[i];
-        bi = lane + 32 * i;
-      }
+  for (int i = 0; i < NV; ++i) {
+    if (((avail >> i) & 1u) && key[i] > bk) {
+      bk = key[i];
+      bi = lane + 32 * i;
     }
   }
-  warp_argbest(bv, bi);
-  if (bi != kNone && (bi & 31) == lane) avail &= ~(1u << (bi >> 5));
+  gk = __reduce_max_sync(0xffffffffu, bk);
+  gi = __reduce_min_sync(0xffffffffu, (bk == gk) ? bi : kNone);
+  if (gi != kNone && (gi & 31) == lane) avail &= ~(1u << (gi >> 5));
 }
 
-__global__ void __launch_bounds__(1024) routing_kernel(RoutingArgs a) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
+__device__ __forceinline__ void cluster_barrier() {
+  __threadfence();
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+__device__ __forceinline__ uint32_t cluster_cta_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+
+// Developer aid: with -DBASE_ROUTING_TIMING the kernel writes %globaltimer stamps of its stages into
+// the buffer passed as dbg.costs (which is then not filled with costs).
+#ifdef BASE_ROUTING_TIMING
+#define RT_STAMP(i)                                                                 \
+  if (gthread == 0 && a.dbg.costs) {                                                \
+    unsigned long long t_;                                                          \
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_));                           \
+    reinterpret_cast<unsigned long long*>(a.dbg.costs)[i] = t_;                     \
+  }
+#else
+#define RT_STAMP(i)
+#endif
+
+template <int NV>
+__global__ void __launch_bounds__(kRoutingThreads) routing_kernel(RoutingArgs a) {
   const int T = a.T, E = a.E, K = a.K, S = T * K;
-  int32_t* s_ids = reinterpret_cast<int32_t*>(smem_raw);      // [S] original routes
-  float* s_cost = reinterpret_cast<float*>(s_ids + S);        // [S] predicted costs, later positions
-  int32_t* s_eids = reinterpret_cast<int32_t*>(s_cost + S);   // [S] executed routes
-  float* s_m = reinterpret_cast<float*>(s_eids + S);          // [T]
-  float* s_S = s_m + T;                                       // [T]
-  float* s_sc = s_S + T;                                      // [E]
-  int32_t* s_cnt = reinterpret_cast<int32_t*>(s_sc + E);      // [E]
-  int32_t* s_off = s_cnt + E;                                 // [E+1]
-  uint8_t* s_mask = reinterpret_cast<uint8_t*>(s_off + E + 1);  // [E]
+  extern __shared__ int32_t s_pos[];   // [S] position of every executed pair inside its expert
+  __shared__ float s_sc[kMaxE];
+  __shared__ int32_t s_cnt[kMaxE];
+  __shared__ int32_t s_off[kMaxE + 1];
+  __shared__ uint8_t s_mask[kMaxE];
+  __shared__ int32_t s_wsum[kRoutingWarps], s_wseg[kRoutingWarps];
   __shared__ int s_status;
 
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
-  const int nv = (E + 31) >> 5;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int cta = int(cluster_cta_rank());
+  const int gwarp = cta * kRoutingWarps + warp;
+  constexpr int kWarps = kClusterCtas * kRoutingWarps;
+  const int gthread = cta * kRoutingThreads + threadIdx.x;
+  constexpr int kAllThreads = kClusterCtas * kRoutingThreads;
   if (threadIdx.x == 0) s_status = 0;
-  __syncthreads();
+  RT_STAMP(0)
 
-  // ---- A: original routes and predicted costs
-  for (int t = warp; t < T; t += nwarp) {
-    float v[kMaxVals];
-    uint32_t avail = 0;
+  // ---- 1: original routes and predicted costs (one warp per token; a lane owns entries lane+32i)
+  for (int t = gwarp; t < T; t += kWarps) {
+    float l[NV], sh[NV];
+    uint32_t key[NV], avail = 0;
+    const float inv_norm = 1.0f / fmaxf(sqrtf(a.znorm2[t]), 1e-30f);
 #pragma unroll
-    for (int i = 0; i < kMaxVals; ++i) {
+    for (int i = 0; i < NV; ++i) {
       const int e = lane + 32 * i;
-      v[i] = -INFINITY;
-      if (i < nv && e < E) {
-        const float l = a.logits[size_t(t) * E + e];
-        v[i] = isnan(l) ? -INFINITY : l;
+      l[i] = -INFINITY;
+      sh[i] = 0.f;
+      if (e < E) {
+        l[i] = a.logits[size_t(t) * E + e];
+        sh[i] = a.raw[size_t(t) * E + e] * inv_norm + a.pred_b[e];
         avail |= 1u << i;
-        a.ws.costs[size_t(t) * E + e] = 0.f;
       }
     }
-    float m = -INFINITY;
 #pragma unroll
-    for (int i = 0; i < kMaxVals; ++i) m = fmaxf(m, v[i]);
-    m = warp_max(m);
-    if (!(m > -INFINITY)) m = 0.f;
-    float S_t = 0.f, myq = 0.f;
+    for (int i = 0; i < NV; ++i) {
+      if (isnan(l[i])) l[i] = -INFINITY;
+      key[i] = float_key(l[i]);
+    }
+    const uint32_t avail0 = avail;
+    float m = 0.f, myv = 0.f;
     int myid = kNone;
     for (int k = 0; k < K; ++k) {
-      float bv;
-      int bi;
-      take_best(v, avail, lane, bv, bi);
-      const float q = (bi == kNone) ? 0.f : expf(bv - m);
-      S_t += q;
+      uint32_t gk;
+      int gi;
+      take_best<NV>(key, avail, lane, gk, gi);
+      const float bv = key_float(gk);
+      if (k == 0) m = (gi != kNone && bv > -INFINITY) ? bv : 0.f;
       if (lane == k) {
-        myq = q;
-        myid = bi;
+        myv = bv;
+        myid = gi;
       }
     }
-    __syncwarp();
+    const uint32_t taken = avail0 & ~avail;
+    float q[NV], qs = 0.f;
+#pragma unroll
+    for (int i = 0; i < NV; ++i) {
+      q[i] = ((taken >> i) & 1u) ? expf(l[i] - m) : 0.f;
+      qs += q[i];
+    }
+    const float S_t = warp_sum(qs);
+#pragma unroll
+    for (int i = 0; i < NV; ++i) {
+      const int e = lane + 32 * i;
+      if (e < E) {
+        float c = 0.f;
+        if ((taken >> i) & 1u) {
+          const float w = S_t > 0.f ? q[i] / S_t : 0.f;
+          c = w * w * expf(sh[i]);
+        }
+        a.ws.costs[size_t(t) * E + e] = c;
+      }
+    }
     if (lane < K) {
       const bool ok = myid != kNone;
-      const float w = (ok && S_t > 0.f) ? myq / S_t : 0.f;
-      float c = 0.f;
-      if (ok) {
-        c = w * w * expf(a.shat[size_t(t) * E + myid]);
-        a.ws.costs[size_t(t) * E + myid] = c;
-      }
+      const float w = (ok && S_t > 0.f) ? expf(myv - m) / S_t : 0.f;
       const int idx = t * K + lane;
-      s_ids[idx] = ok ? myid : -1;
-      s_cost[idx] = c;
       a.ws.topk_ids[idx] = ok ? myid : -1;
       a.ws.topk_w[idx] = w;
       if (a.dbg.topk_ids) a.dbg.topk_ids[idx] = ok ? myid : -1;
       if (a.dbg.topk_w) a.dbg.topk_w[idx] = w;
     }
     if (lane == 0) {
-      s_m[t] = m;
-      s_S[t] = S_t;
+      a.ws.tok_m[t] = m;
+      a.ws.tok_S[t] = S_t;
     }
   }
-  __syncthreads();
-  if (a.dbg.costs) {
-    for (int i = threadIdx.x; i < T * E; i += blockDim.x) a.dbg.costs[i] = a.ws.costs[i];
-  }
-  if (a.dbg.logits) {
-    for (int i = threadIdx.x; i < T * E; i += blockDim.x) a.dbg.logits[i] = a.logits[i];
-  }
+  RT_STAMP(1)
+  cluster_barrier();
+  RT_STAMP(2)
 
-  // ---- B: batch aggregation, fixed order (see aggregate_select_kernel)
-  for (int e = warp; e < E; e += nwarp) {
-    float acc = 0.f;
-    for (int t = lane; t < T; t += 32) {
-      float c = 0.f;
-      for (int k = 0; k < K; ++k)
-        if (s_ids[t * K + k] == e) c = s_cost[t * K + k];
-      acc += c;
-    }
-    acc = warp_sum(acc);
-    if (lane == 0) {
-      int nf = 0;
-      s_sc[e] = sortable(acc, &nf);
-      if (nf) atomicOr(&s_status, BASE_DEV_NONFINITE_SCORE);
-      a.ws.scores[e] = acc;
-      if (a.dbg.scores) a.dbg.scores[e] = acc;
-    }
-  }
-  __syncthreads();
-
-  // ---- C: top-M by rank counting
-  const int M = min(a.M, E);
-  for (int e = threadIdx.x; e < E; e += blockDim.x) {
-    const int r = rank_of(s_sc, E, e);
-    const uint8_t in = r < M;
-    a.ws.mask[e] = in;
-    if (in) a.ws.selected[r] = e;
-    if (a.dbg.active_mask) a.dbg.active_mask[e] = in;
-    if (in && a.dbg.selected_ids) a.dbg.selected_ids[r] = e;
-    s_mask[e] = a.forced_mask ? (a.forced_mask[e] != 0) : in;
-    s_cnt[e] = 0;
-  }
-  __syncthreads();
-
-  // ---- D: restricted routes and gates
-  for (int t = warp; t < T; t += nwarp) {
-    float v[kMaxVals];
-    uint32_t avail = 0;
+  // ---- 2: batch aggregation in a fixed order (lane l adds tokens l, l+32, ... ascending, then an
+  // xor tree: the order of aggregate_select_kernel). Every CTA sums all experts itself (the costs are
+  // a few KB in L2), eight experts per warp at a time so that their loads are in flight together.
+  for (int e0 = warp; e0 < E; e0 += kRoutingWarps * 8) {
+    float acc[8];
 #pragma unroll
-    for (int i = 0; i < kMaxVals; ++i) {
+    for (int j = 0; j < 8; ++j) acc[j] = 0.f;
+#pragma unroll 2
+    for (int t = lane; t < T; t += 32) {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const int e = e0 + j * kRoutingWarps;
+        if (e < E) acc[j] += a.ws.costs[size_t(t) * E + e];
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc[j] = warp_sum(acc[j]);
+    if (lane == 0) {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const int e = e0 + j * kRoutingWarps;
+        if (e < E) {
+          int nf = 0;
+          s_sc[e] = sortable(acc[j], &nf);
+          if (nf) atomicOr(&s_status, BASE_DEV_NONFINITE_SCORE);
+          if (cta == 0) {
+            a.ws.scores[e] = acc[j];
+            if (a.dbg.scores) a.dbg.scores[e] = acc[j];
+          }
+        }
+      }
+    }
+  }
+#ifndef BASE_ROUTING_TIMING
+  if (a.dbg.costs)
+    for (int i = gthread; i < T * E; i += kAllThreads) a.dbg.costs[i] = a.ws.costs[i];
+#endif
+  if (a.dbg.logits)
+    for (int i = gthread; i < T * E; i += kAllThreads) a.dbg.logits[i] = a.logits[i];
+  __syncthreads();
+  RT_STAMP(3)
+
+  // ---- 3: top-M by rank counting (every CTA keeps its own copy of the active mask): four threads
+  // per expert each count a quarter of the experts that come before it (score desc, id asc) ...
+  const int M = min(a.M, E);
+  for (int e0 = 0; e0 < E; e0 += kRoutingThreads / 4) {
+    const int e = e0 + (threadIdx.x >> 2), part = threadIdx.x & 3;
+    int r = 0;
+    if (e < E) {
+      const float se = s_sc[e];
+#pragma unroll 4
+      for (int j = part; j < E; j += 4) {
+        const float sj = s_sc[j];
+        r += (sj > se) || (sj == se && j < e);
+      }
+    }
+    r += __shfl_xor_sync(0xffffffffu, r, 1);
+    r += __shfl_xor_sync(0xffffffffu, r, 2);
+    if (e < E && part == 0) {
+      const uint8_t in = r < M;
+      s_mask[e] = a.forced_mask ? (a.forced_mask[e] != 0) : in;
+      if (cta == 0) {
+        a.ws.mask[e] = in;
+        if (in) a.ws.selected[r] = e;
+        if (a.dbg.active_mask) a.dbg.active_mask[e] = in;
+        if (in && a.dbg.selected_ids) a.dbg.selected_ids[r] = e;
+      }
+    }
+  }
+  for (int e = threadIdx.x; e < E; e += kRoutingThreads) s_cnt[e] = 0;
+  __syncthreads();
+  RT_STAMP(4)
+
+  // ---- ... and the restricted routes of this CTA's tokens
+  for (int t = gwarp; t < T; t += kWarps) {
+    uint32_t key[NV], avail = 0;
+    const float m = a.ws.tok_m[t], S_t = a.ws.tok_S[t];
+#pragma unroll
+    for (int i = 0; i < NV; ++i) {
       const int e = lane + 32 * i;
-      v[i] = -INFINITY;
-      if (i < nv && e < E) {
-        const float l = a.logits[size_t(t) * E + e];
-        v[i] = isnan(l) ? -INFINITY : l;
+      key[i] = 0;
+      if (e < E) {
+        const float lv = a.logits[size_t(t) * E + e];
+        key[i] = float_key(isnan(lv) ? -INFINITY : lv);
         bool ok = s_mask[e] != 0;
         if (ok && a.fill_rule == BASE_FILL_DROP) {
           ok = false;
-          for (int k = 0; k < K; ++k) ok |= (s_ids[t * K + k] == e);
+          for (int k = 0; k < K; ++k) ok |= (a.ws.topk_ids[t * K + k] == e);
         }
         if (ok) avail |= 1u << i;
       }
     }
-    const float m = s_m[t];
-    float sumq = 0.f, myq = 0.f;
+    float myq = 0.f;
     int myid = kNone;
     for (int k = 0; k < K; ++k) {
-      float bv;
-      int bi;
-      take_best(v, avail, lane, bv, bi);
-      const float q = (bi == kNone) ? 0.f : expf(bv - m);
-      sumq += q;
+      uint32_t gk;
+      int gi;
+      take_best<NV>(key, avail, lane, gk, gi);
       if (lane == k) {
-        myq = q;
-        myid = bi;
+        myid = gi;
+        myq = (gi != kNone) ? expf(key_float(gk) - m) : 0.f;
       }
     }
+    const float sumq = warp_sum(myq);
     if (lane < K) {
-      const float den = (a.gate_rule == BASE_GATE_RENORM) ? sumq : s_S[t];
+      const float den = (a.gate_rule == BASE_GATE_RENORM) ? sumq : S_t;
       const bool ok = myid != kNone;
       const float g = (ok && den > 0.f) ? myq / den : 0.f;
       const int idx = t * K + lane;
-      s_eids[idx] = ok ? myid : -1;
       a.ws.exec_ids[idx] = ok ? myid : -1;
       a.ws.exec_gates[idx] = g;
       if (a.dbg.exec_ids) a.dbg.exec_ids[idx] = ok ? myid : -1;
       if (a.dbg.exec_gates) a.dbg.exec_gates[idx] = g;
     }
   }
-  __syncthreads();
+  RT_STAMP(5)
+  cluster_barrier();
+  RT_STAMP(6)
 
-  // ---- E: dispatch lists. Position of a pair inside its expert = number of lower-numbered tokens
-  // routed to that expert, so each expert's rows are in token order.
-  int32_t* s_pos = reinterpret_cast<int32_t*>(s_cost);
-  for (int e = warp; e < E; e += nwarp) {
-    int base_cnt = 0;
-    for (int t0 = 0; t0 < T; t0 += 32) {
-      const int t = t0 + lane;
+  // ---- 4: dispatch lists, computed by every CTA. A warp owns the experts e = warp (mod 16); a lane
+  // holds one token's executed routes in registers. Position of a pair inside its expert = number of
+  // lower-numbered tokens routed to that expert, so each expert's rows are in token order.
+  for (int t0 = 0; t0 < T; t0 += 32) {
+    const int t = t0 + lane;
+    int ids[kMaxK];
+#pragma unroll
+    for (int k = 0; k < kMaxK; ++k) ids[k] = (t < T && k < K) ? a.ws.exec_ids[t * K + k] : -1;
+    for (int e = warp; e < E; e += kRoutingWarps) {
       int kk = -1;
-      if (t < T) {
-        for (int k = 0; k < K; ++k)
-          if (s_eids[t * K + k] == e) kk = k;
-      }
+#pragma unroll
+      for (int k = 0; k < kMaxK; ++k)
+        if (ids[k] == e) kk = k;
       const uint32_t bal = __ballot_sync(0xffffffffu, kk >= 0);
-      if (kk >= 0) s_pos[t * K + kk] = base_cnt + __popc(bal & ((1u << lane) - 1u));
-      base_cnt += __popc(bal);
+      if (bal) {
+        const int base_cnt = s_cnt[e];
+        if (kk >= 0) s_pos[t * K + kk] = base_cnt + __popc(bal & ((1u << lane) - 1u));
+        __syncwarp();
+        if (lane == 0) s_cnt[e] = base_cnt + __popc(bal);
+      }
     }
-    if (lane == 0) s_cnt[e] = base_cnt;
+    __syncwarp();
   }
   __syncthreads();
-  if (warp == 0) {
-    // exclusive scan of the counts, the compact list of dispatched experts, and the work segments
-    int run = 0, nseg = 0, ndisp = 0;
-    for (int e0 = 0; e0 < E; e0 += 32) {
-      const int e = e0 + lane;
-      const int c = (e < E) ? s_cnt[e] : 0;
-      const int segs = (c + kSegTokens - 1) / kSegTokens;
-      int incl = c, sincl = segs;
+  RT_STAMP(7)
+  // exclusive scan of the counts (and of the per-expert segment counts) over the block
+  {
+    const int e = threadIdx.x;   // E <= kRoutingThreads
+    const int c = (e < E) ? s_cnt[e] : 0;
+    const int segs = (c + kSegTokens - 1) / kSegTokens;
+    int incl = c, sincl = segs;
 #pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const int x = __shfl_up_sync(0xffffffffu, incl, o);
-        const int y = __shfl_up_sync(0xffffffffu, sincl, o);
-        if (lane >= o) {
-          incl += x;
-          sincl += y;
-        }
+    for (int o = 1; o < 32; o <<= 1) {
+      const int x = __shfl_up_sync(0xffffffffu, incl, o);
+      const int y = __shfl_up_sync(0xffffffffu, sincl, o);
+      if (lane >= o) {
+        incl += x;
+        sincl += y;
       }
-      const int off = run + incl - c;
-      if (e < E) {
-        s_off[e] = off;
+    }
+    if (lane == 31) {
+      s_wsum[warp] = incl;
+      s_wseg[warp] = sincl;
+    }
+    const int ndisp = __syncthreads_count(c > 0);
+    int run = 0, nseg = 0;
+#pragma unroll
+    for (int w = 0; w < kRoutingWarps; ++w) {
+      if (w < warp) {
+        run += s_wsum[w];
+        nseg += s_wseg[w];
+      }
+    }
+    const int off = run + incl - c;
+    if (e < E) {
+      s_off[e] = off;
+      if (cta == 0) {
         a.ws.expert_offset[e] = off;
         a.ws.expert_count[e] = c;
+        a.ws.counters[kCtrReady + e] = 0;
         if (a.dbg.expert_counts) a.dbg.expert_counts[e] = c;
-        for (int s = 0; s < segs; ++s) {
-          const int si = nseg + sincl - segs + s;
+        for (int sgi = 0; sgi < segs; ++sgi) {
+          const int si = nseg + sincl - segs + sgi;
           a.ws.seg_expert[si] = e;
-          a.ws.seg_offset[si] = off + s * kSegTokens;
-          a.ws.seg_count[si] = min(kSegTokens, c - s * kSegTokens);
+          a.ws.seg_offset[si] = off + sgi * kSegTokens;
+          a.ws.seg_count[si] = min(kSegTokens, c - sgi * kSegTokens);
         }
       }
-      ndisp += __popc(__ballot_sync(0xffffffffu, c > 0));
-      run += __shfl_sync(0xffffffffu, incl, 31);
-      nseg += __shfl_sync(0xffffffffu, sincl, 31);
     }
-    if (lane == 0) {
-      s_off[E] = run;
-      a.ws.expert_offset[E] = run;
+    if (e == E - 1 && cta == 0) {
+      a.ws.expert_offset[E] = off + c;
       a.ws.counters[kCtrDispatched] = ndisp;
-      a.ws.counters[kCtrSegments] = nseg;
-      a.ws.counters[kCtrSlots] = run;
+      a.ws.counters[kCtrSegments] = nseg + sincl;
+      a.ws.counters[kCtrSlots] = off + c;
+      a.ws.counters[kCtrStatus] = s_status;
+      a.ws.counters[kCtrTicket] = 0;
       if (a.dbg.n_dispatched) a.dbg.n_dispatched[0] = ndisp;
+      if (a.dbg.status) a.dbg.status[0] = s_status;
     }
   }
   __syncthreads();
-  for (int i = threadIdx.x; i < S; i += blockDim.x) {
-    const int e = s_eids[i];
+  RT_STAMP(8)
+  for (int i = gthread; i < S; i += kAllThreads) {
+    const int e = a.ws.exec_ids[i];
     int slot = -1;
     if (e >= 0) {
       slot = s_off[e] + s_pos[i];
@@ -458,57 +606,80 @@ __global__ void __launch_bounds__(1024) routing_kernel(RoutingArgs a) {
     }
     a.ws.token_slot[i] = slot;
   }
-  for (int e = threadIdx.x; e < E; e += blockDim.x) a.ws.counters[kCtrReady + e] = 0;
-  if (threadIdx.x == 0) {
-    a.ws.counters[kCtrStatus] = s_status;
-    a.ws.counters[kCtrTicket] = 0;
-    if (a.dbg.status) a.dbg.status[0] = s_status;
-  }
+  RT_STAMP(9)
 }
 
-size_t routing_smem_bytes(int T, int E, int K) {
-  const size_t S = size_t(T) * K;
-  return 3 * S * 4 + 2 * size_t(T) * 4 + size_t(E) * 4 + size_t(E) * 4 + size_t(E + 1) * 4 + size_t(E) + 16;
+constexpr size_t kRoutingMaxSmem = size_t(kMaxSlots) * 4;
+
+template <int NV>
+cudaError_t launch_routing_nv(const RoutingArgs& a, cudaLaunchConfig_t* cfg) {
+  static cudaError_t attr = cudaFuncSetAttribute(routing_kernel<NV>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                 int(kRoutingMaxSmem));
+  if (attr != cudaSuccess) return attr;
+  return cudaLaunchKernelEx(cfg, routing_kernel<NV>, a);
 }
 
 cudaError_t launch_routing(const RoutingArgs& a, cudaStream_t st) {
-  const size_t smem = routing_smem_bytes(a.T, a.E, a.K);
-  static thread_local size_t configured = 0;
-  if (smem > 48 * 1024 && smem > configured) {
-    cudaError_t e = cudaFuncSetAttribute(routing_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
-    if (e != cudaSuccess) return e;
-    configured = smem;
-  }
-  int threads = 32 * max(4, min(32, max(a.T, (a.E + 31) / 32)));
-  routing_kernel<<<1, threads, smem, st>>>(a);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(kClusterCtas);
+  cfg.blockDim = dim3(kRoutingThreads);
+  cfg.dynamicSmemBytes = size_t(a.T) * a.K * 4;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = kClusterCtas;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  const int nv = (a.E + 31) / 32;
+  if (nv <= 1) return launch_routing_nv<1>(a, &cfg);
+  if (nv <= 2) return launch_routing_nv<2>(a, &cfg);
+  if (nv <= 4) return launch_routing_nv<4>(a, &cfg);
+  if (nv <= 8) return launch_routing_nv<8>(a, &cfg);
+  return launch_routing_nv<16>(a, &cfg);
 }
 
 // ------------------------------------------------------------------------------------------------
-// Gather the token inputs into expert-sorted order: x_sorted[slot] = hidden[slot_token[slot]].
+// Gather the token inputs into expert-sorted order: x_sorted[row] = hidden[slot_token[row]].
+// One warp per row, all 16-byte loads of a row in flight before the first store.
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) gather_kernel(const __nv_bfloat16* __restrict__ hidden,
                                                      const int32_t* __restrict__ slot_token,
                                                      const int32_t* __restrict__ counters,
                                                      __nv_bfloat16* __restrict__ x_sorted, int d) {
-  const int slot = blockIdx.x;
+  const int slot = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
   if (slot >= counters[kCtrSlots]) return;
   const int t = slot_token[slot];
   const uint4* src = reinterpret_cast<const uint4*>(hidden + size_t(t) * d);
   uint4* dst = reinterpret_cast<uint4*>(x_sorted + size_t(slot) * d);
-  for (int j = threadIdx.x; j < (d >> 3); j += blockDim.x) dst[j] = __ldg(src + j);
+  const int dv = d >> 3;
+  for (int j0 = 0; j0 < dv; j0 += 256) {
+    uint4 v[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int j = j0 + i * 32 + lane;
+      if (j < dv) v[i] = __ldg(src + j);
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int j = j0 + i * 32 + lane;
+      if (j < dv) dst[j] = v[i];
+    }
+  }
 }
 
 cudaError_t launch_gather(const void* hidden, const Workspace& ws, int T, int K, int d, cudaStream_t st) {
-  gather_kernel<<<T * K, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(hidden), ws.slot_token, ws.counters,
-                                       ws.x_sorted, d);
+  gather_kernel<<<(T * K + 7) / 8, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(hidden), ws.slot_token, ws.counters,
+                                                 ws.x_sorted, d);
   return cudaGetLastError();
 }
 
 // ------------------------------------------------------------------------------------------------
 // Combine: y[t] = sum_k gate[t,k] * ypair[row(t,k)] in slot order k = 0..K-1 (deterministic).
 // With x_next != nullptr also writes rmsnorm(hidden[t] + y[t]) (no gain) as bf16: the wiring
-// between consecutive layers of the stack workload.
+// between consecutive layers of the stack workload. One CTA per token; the K row reads of a column
+// group are issued together.
 // ------------------------------------------------------------------------------------------------
 constexpr int kCombineIters = 8;  // d <= 256 threads * 4 * 8 = 8192
 
@@ -522,9 +693,10 @@ __global__ void __launch_bounds__(256) combine_kernel(const float* __restrict__ 
   __shared__ int s_slot[kMaxK];
   __shared__ float s_gate[kMaxK];
   __shared__ float s_red[8];
-  if (threadIdx.x < K) {
-    s_slot[threadIdx.x] = token_slot[t * K + threadIdx.x];
-    s_gate[threadIdx.x] = gates[t * K + threadIdx.x];
+  if (threadIdx.x < kMaxK) {
+    const bool in = threadIdx.x < K;
+    s_slot[threadIdx.x] = in ? token_slot[t * K + threadIdx.x] : -1;
+    s_gate[threadIdx.x] = in ? gates[t * K + threadIdx.x] : 0.f;
   }
   __syncthreads();
   float4 keep[kCombineIters];
@@ -533,16 +705,22 @@ __global__ void __launch_bounds__(256) combine_kernel(const float* __restrict__ 
   for (int it = 0; it < kCombineIters; ++it) {
     const int c = (it * 256 + threadIdx.x) * 4;
     if (c >= d) break;
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int k = 0; k < K; ++k) {
+    float4 v[kMaxK];
+#pragma unroll
+    for (int k = 0; k < kMaxK; ++k) {
       const int slot = s_slot[k];
-      if (slot < 0) continue;
-      const float g = s_gate[k];
-      const float4 v = *reinterpret_cast<const float4*>(ypair + size_t(slot) * d + c);
-      acc.x = fmaf(g, v.x, acc.x);
-      acc.y = fmaf(g, v.y, acc.y);
-      acc.z = fmaf(g, v.z, acc.z);
-      acc.w = fmaf(g, v.w, acc.w);
+      v[k] = slot >= 0 ? *reinterpret_cast<const float4*>(ypair + size_t(slot) * d + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int k = 0; k < kMaxK; ++k) {
+      if (s_slot[k] >= 0) {
+        const float g = s_gate[k];
+        acc.x = fmaf(g, v[k].x, acc.x);
+        acc.y = fmaf(g, v[k].y, acc.y);
+        acc.z = fmaf(g, v[k].z, acc.z);
+        acc.w = fmaf(g, v[k].w, acc.w);
+      }
     }
     if (out) {
       if (out_is_fp32) {
