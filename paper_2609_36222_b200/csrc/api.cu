@@ -68,6 +68,7 @@ int enqueue_layer(const LayerCall& c, const Workspace& ws, cudaStream_t st, int*
   ra.forced_mask = c.forced_mask;
   ra.hidden = static_cast<const __nv_bfloat16*>(c.hidden);
   ra.d = s.d;
+  ra.max_segs = max_segments(s.E, c.T, s.K);
   ra.T = c.T;
   ra.E = s.E;
   ra.K = s.K;

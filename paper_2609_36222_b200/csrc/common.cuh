@@ -65,7 +65,7 @@ struct Workspace {
   int32_t* seg_count;     // [max_segs]
   float* tok_m;           // [T] max logit of the token
   float* tok_S;           // [T] softmax denominator over the original top-K
-  int32_t* counters;      // [16 + E]: 0 n_dispatched, 1 n_segments, 2 status, 3 total slots, 4.. tickets; 16.. per-expert ready
+  int32_t* counters;      // [16 + max_segs]: 0 n_dispatched, 1 n_segments, 2 status, 3 total slots, 4 ticket; 16.. per-segment count of finished gate/up tiles
   __nv_bfloat16* x_sorted; // [T*K + pad, d] token inputs in expert-sorted order
   __nv_bfloat16* h;        // [T*K + pad, I] silu(gate) * up, expert-sorted
   float* ypair;            // [T*K, d] down-projection outputs per routed pair
@@ -117,7 +117,7 @@ inline Workspace carve_workspace(void* base_ptr, const base_layer_shape& s, int 
   w.seg_count = static_cast<int32_t*>(take(size_t(segs) * 4, 256));
   w.tok_m = static_cast<float*>(take(size_t(T) * 4, 256));
   w.tok_S = static_cast<float*>(take(size_t(T) * 4, 256));
-  w.counters = static_cast<int32_t*>(take(size_t(kCtrReady + s.E) * 4, 256));
+  w.counters = static_cast<int32_t*>(take(size_t(kCtrReady + segs) * 4, 256));
   w.bytes = align_up(off, 1024);
   return w;
 }
@@ -131,7 +131,7 @@ struct RoutingArgs {
   const float* pred_b;        // [E]
   const uint8_t* forced_mask; // or nullptr
   const __nv_bfloat16* hidden; // [T,d] token inputs (gathered into expert-sorted order)
-  int T, E, K, M, d, gate_rule, fill_rule;
+  int T, E, K, M, d, gate_rule, fill_rule, max_segs;
   Workspace ws;
   base_layer_debug dbg;       // zero-initialised when the caller passed none
 };

@@ -82,10 +82,9 @@ struct FfnParams {
   int32_t* counters;
   __nv_bfloat16* h;     // gate/up pass output
   float* ypair;         // down pass output
-  int rows_per_expert;  // I (gate/up) or d (down): rows of one expert in the weight tensor map
-  int tiles;            // work units per segment
-  int kblocks;          // K extent / 64
   int I, d;
+  int tiles1, tiles2;   // work units per segment: I/64 gate/up tiles, d/128 down tiles
+  int steps1, steps2;   // pipeline stages per unit: ceil(d/64 / 2), ceil(I/64 / 2)
   int split_a;          // gate/up pass: 1 = gate and up come from two maps (two boxes per k-block)
 };
 
@@ -211,14 +210,23 @@ __device__ __forceinline__ bool named_and(int id, int threads, bool pred) {
   return out != 0;
 }
 
+// Work units of one launch, in execution order: all gate/up tiles (segment-major), then all down
+// tiles. CTA c takes units c, c + grid, c + 2 grid, ...: every CTA finishes its gate/up units before
+// it touches a down unit, so the dependency of a down unit (all gate/up tiles of its segment) is
+// always on work that never waits itself.
 struct Unit {
-  int expert, offset, count, npad, tile;
+  int phase, seg, expert, offset, count, npad, tile;
 };
 
-__device__ __forceinline__ Unit decode_unit(const FfnParams& p, int u) {
+__device__ __forceinline__ Unit decode_unit(const FfnParams& p, int u, int n_seg) {
   Unit r;
-  const int seg = u / p.tiles;
-  r.tile = u - seg * p.tiles;
+  const int u1 = n_seg * p.tiles1;
+  r.phase = u < u1 ? 1 : 2;
+  const int v = u < u1 ? u : u - u1;
+  const int tiles = u < u1 ? p.tiles1 : p.tiles2;
+  const int seg = v / tiles;
+  r.seg = seg;
+  r.tile = v - seg * tiles;
   r.expert = p.seg_expert[seg];
   r.offset = p.seg_offset[seg];
   r.count = p.seg_count[seg];
@@ -227,8 +235,18 @@ __device__ __forceinline__ Unit decode_unit(const FfnParams& p, int u) {
 }
 
 // ------------------------------------------------------------------------------------------- the kernel
-template <int kPhase, int kMaxN>
-__global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_constant__ MapSet maps, const FfnParams p) {
+__device__ __forceinline__ int ld_acquire(const int32_t* ptr) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(ptr) : "memory");
+  return v;
+}
+__device__ __forceinline__ void red_release_add(int32_t* ptr, int v) {
+  asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(ptr), "r"(v) : "memory");
+}
+
+template <int kMaxN>
+__global__ void __launch_bounds__(kThreads, 1)
+ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapSet maps2, const FfnParams p) {
   using P = Plan<kMaxN>;
   constexpr int kStages = P::kStages, kStageBytes = P::kStageBytes, kAccCols = P::kAccCols, kTmemCols = P::kTmemCols;
   constexpr int kStageABytes = kKbPerStage * kTileABytes;
@@ -240,8 +258,9 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
   volatile int* abort_flag = &bars->abort_flag;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n_units = p.counters[kCtrSegments] * p.tiles;
-  const int n_steps = (p.kblocks + kKbPerStage - 1) / kKbPerStage;   // pipeline stages per unit
+  const int n_seg = p.counters[kCtrSegments];
+  const int n_units = n_seg * (p.tiles1 + p.tiles2);
+  const int kblocks1 = p.d / kBlockK, kblocks2 = p.I / kBlockK;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
@@ -254,8 +273,9 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
     }
     bars->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("prefetch.tensormap [%0];" ::"l"(&maps.a) : "memory");
-    if (kPhase == 1 && p.split_a) asm volatile("prefetch.tensormap [%0];" ::"l"(&maps.a2) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&maps1.a) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&maps2.a) : "memory");
+    if (p.split_a) asm volatile("prefetch.tensormap [%0];" ::"l"(&maps1.a2) : "memory");
   }
   if (warp == 1) tmem_alloc(smem_u32(&bars->tmem_base), kTmemCols);
   tcgen05_fence_before();
@@ -270,10 +290,13 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
       uint32_t phase = 0;
       bool ok = true;
       for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
-        const Unit un = decode_unit(p, u);
-        const int arow = un.expert * p.rows_per_expert + un.tile * (kPhase == 1 ? 64 : 128);
-        const CUtensorMap* tm_b = &maps.b[(un.npad >> 4) - 1];
+        const Unit un = decode_unit(p, u, n_seg);
+        const bool gu = un.phase == 1;
+        const int arow = gu ? un.expert * p.I + un.tile * 64 : un.expert * p.d + un.tile * 128;
+        const CUtensorMap* tm_b = gu ? &maps1.b[(un.npad >> 4) - 1] : &maps2.b[(un.npad >> 4) - 1];
         const uint32_t bytes = uint32_t(kKbPerStage * (kTileABytes + un.npad * 128));
+        const int n_steps = gu ? p.steps1 : p.steps2;
+        bool h_ready = gu;   // a down unit reads h rows that other CTAs write
         for (int st = 0; st < n_steps; ++st) {
           if (!mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1u, abort_flag)) {
             ok = false;
@@ -286,18 +309,41 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
           // k-blocks past the end of K are out of the tensor's bounds and arrive as zeros; the box
           // always delivers its full byte count.
           mbar_expect_tx(full, bytes);
-          if (kPhase == 1) {
+          if (gu) {
             if (!p.split_a) {
-              tma_load_4d(sa, &maps.a, 0, arow, 0, kb, full);      // {elem, row, gate|up, k-block}
+              tma_load_4d(sa, &maps1.a, 0, arow, 0, kb, full);      // {elem, row, gate|up, k-block}
             } else {
 #pragma unroll
               for (int j = 0; j < kKbPerStage; ++j) {
-                tma_load_3d(sa + j * kTileABytes, &maps.a, 0, arow, kb + j, full);
-                tma_load_3d(sa + j * kTileABytes + kTileABytes / 2, &maps.a2, 0, arow, kb + j, full);
+                tma_load_3d(sa + j * kTileABytes, &maps1.a, 0, arow, kb + j, full);
+                tma_load_3d(sa + j * kTileABytes + kTileABytes / 2, &maps1.a2, 0, arow, kb + j, full);
               }
             }
           } else {
-            tma_load_3d(sa, &maps.a, 0, arow, kb, full);             // {elem, row, k-block}
+            tma_load_3d(sa, &maps2.a, 0, arow, kb, full);            // {elem, row, k-block}
+          }
+          if (!h_ready) {
+            // The weight box above is already in flight; now wait (bounded) until every gate/up tile
+            // of this segment has published its h rows.
+            const int32_t* flag = p.counters + kCtrReady + un.seg;
+            const long long t0 = clock64();
+            bool ready = false;
+#pragma unroll 1
+            for (uint32_t it = 0; it < kSpinLimit; ++it) {
+              if (ld_acquire(flag) >= p.tiles1) {
+                ready = true;
+                break;
+              }
+              __nanosleep(64);
+              if ((it & 255u) == 255u && (*abort_flag || clock64() - t0 > kWaitCycles)) break;
+            }
+            if (!ready) {
+              *abort_flag = 1;
+              ok = false;
+              break;
+            }
+            asm volatile("fence.proxy.async;" ::: "memory");   // generic-proxy writes -> async-proxy (TMA) reads
+            h_ready = true;
           }
           tma_load_3d(sb, tm_b, 0, un.offset, kb, full);
           if (++stage == kStages) {
@@ -315,7 +361,9 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
       uint32_t phase = 0, acc_phase = 0;
       bool ok = true;
       for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
-        const Unit un = decode_unit(p, u);
+        const Unit un = decode_unit(p, u, n_seg);
+        const int n_steps = un.phase == 1 ? p.steps1 : p.steps2;
+        const int kblocks = un.phase == 1 ? kblocks1 : kblocks2;
         if (!mbar_wait(smem_u32(&bars->acc_empty[acc]), acc_phase ^ 1u, abort_flag)) break;
         tcgen05_fence_after();
         const uint32_t d_tmem = tmem_base + uint32_t(acc * kAccCols);
@@ -331,7 +379,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
           const uint32_t sb = sa + kStageABytes;
 #pragma unroll
           for (int j = 0; j < kKbPerStage; ++j) {
-            if (st * kKbPerStage + j < p.kblocks) {
+            if (st * kKbPerStage + j < kblocks) {
               const uint64_t adesc = make_smem_desc(sa + j * kTileABytes);
               const uint64_t bdesc = make_smem_desc(sb + j * tile_b);
 #pragma unroll
@@ -358,14 +406,14 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
     int acc = 0;
     uint32_t acc_phase = 0;
     for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
-      const Unit un = decode_unit(p, u);
+      const Unit un = decode_unit(p, u, n_seg);
       int got = 0;
       if (lane == 0) got = mbar_wait(smem_u32(&bars->acc_full[acc]), acc_phase, abort_flag, 128) ? 1 : 0;
       got = __shfl_sync(0xffffffffu, got, 0);
       if (!named_and(1, 128, got != 0)) break;
       tcgen05_fence_after();
       const uint32_t taddr = tmem_base + (uint32_t(q * 32) << 16) + uint32_t(acc * kAccCols);
-      if (kPhase == 1) {
+      if (un.phase == 1) {
         const int r = (q & 1) * 32 + lane;  // row inside the 64-row slice
         if (q >= 2) {
           // up rows: park them in shared memory for the gate warps
@@ -397,6 +445,10 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
           }
           tcgen05_fence_before();
           mbar_arrive(smem_u32(&bars->acc_empty[acc]));
+          // publish: this tile's h rows are complete once all 64 gate threads have fenced their stores
+          __threadfence();
+          named_sync(4, 64);
+          if (q == 0 && lane == 0) red_release_add(p.counters + kCtrReady + un.seg, 1);
         }
       } else {
         float* yrow = p.ypair + size_t(un.offset) * p.d + un.tile * 128 + q * 32 + lane;
@@ -558,33 +610,13 @@ int sm_count() {
   return n;
 }
 
-template <int kPhase, int kMaxN>
-cudaError_t configure() {
-  static cudaError_t st = cudaFuncSetAttribute(ffn_tc_kernel<kPhase, kMaxN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                               int(Plan<kMaxN>::kSmemBytes));
-  return st;
-}
-
 template <int kMaxN>
-cudaError_t launch_both(const MapSet& m1, const MapSet& m2, FfnParams p, const base_layer_shape& s, int segs,
-                        cudaStream_t st) {
-  cudaError_t e = configure<1, kMaxN>();
-  if (e != cudaSuccess) return e;
-  e = configure<2, kMaxN>();
-  if (e != cudaSuccess) return e;
-  p.rows_per_expert = s.I;
-  p.tiles = s.I / 64;
-  p.kblocks = s.d / kBlockK;
-  int grid = min(sm_count(), segs * p.tiles);
-  ffn_tc_kernel<1, kMaxN><<<grid, kThreads, Plan<kMaxN>::kSmemBytes, st>>>(m1, p);
-  e = cudaGetLastError();
-  if (e != cudaSuccess) return e;
-  p.rows_per_expert = s.d;
-  p.tiles = s.d / 128;
-  p.kblocks = s.I / kBlockK;
-  p.split_a = 0;
-  grid = min(sm_count(), segs * p.tiles);
-  ffn_tc_kernel<2, kMaxN><<<grid, kThreads, Plan<kMaxN>::kSmemBytes, st>>>(m2, p);
+cudaError_t launch_kernel(const MapSet& m1, const MapSet& m2, const FfnParams& p, int max_units, cudaStream_t st) {
+  static cudaError_t attr = cudaFuncSetAttribute(ffn_tc_kernel<kMaxN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                 int(Plan<kMaxN>::kSmemBytes));
+  if (attr != cudaSuccess) return attr;
+  const int grid = min(sm_count(), max_units);
+  ffn_tc_kernel<kMaxN><<<grid, kThreads, Plan<kMaxN>::kSmemBytes, st>>>(m1, m2, p);
   return cudaGetLastError();
 }
 
@@ -619,12 +651,17 @@ cudaError_t launch_ffn_tc(const base_layer_shape& s, const base_layer_weights& w
   p.ypair = ws.ypair;
   p.I = s.I;
   p.d = s.d;
+  p.tiles1 = s.I / 64;
+  p.tiles2 = s.d / 128;
+  p.steps1 = (s.d / kBlockK + kKbPerStage - 1) / kKbPerStage;
+  p.steps2 = (s.I / kBlockK + kKbPerStage - 1) / kKbPerStage;
+  const int max_units = segs * (p.tiles1 + p.tiles2);
   // No expert can receive more tokens than the batch holds, which bounds the token tile.
   cudaError_t e;
-  if (T <= 32) e = launch_both<32>(m1, m2, p, s, segs, st);
-  else if (T <= 64) e = launch_both<64>(m1, m2, p, s, segs, st);
-  else e = launch_both<128>(m1, m2, p, s, segs, st);
-  *launches += 2;
+  if (T <= 32) e = launch_kernel<32>(m1, m2, p, max_units, st);
+  else if (T <= 64) e = launch_kernel<64>(m1, m2, p, max_units, st);
+  else e = launch_kernel<128>(m1, m2, p, max_units, st);
+  *launches += 1;
   return e;
 }
 

@@ -574,7 +574,6 @@ __global__ void __launch_bounds__(kRoutingThreads) routing_kernel(RoutingArgs a)
       if (cta == 0) {
         a.ws.expert_offset[e] = off;
         a.ws.expert_count[e] = c;
-        a.ws.counters[kCtrReady + e] = 0;
         if (a.dbg.expert_counts) a.dbg.expert_counts[e] = c;
         for (int sgi = 0; sgi < segs; ++sgi) {
           const int si = nseg + sincl - segs + sgi;
@@ -597,6 +596,8 @@ __global__ void __launch_bounds__(kRoutingThreads) routing_kernel(RoutingArgs a)
   }
   __syncthreads();
   RT_STAMP(8)
+  if (cta == 0)
+    for (int i = threadIdx.x; i < a.max_segs; i += kRoutingThreads) a.ws.counters[kCtrReady + i] = 0;
   for (int i = gthread; i < S; i += kAllThreads) {
     const int e = a.ws.exec_ids[i];
     int slot = -1;
