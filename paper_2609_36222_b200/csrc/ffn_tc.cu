@@ -258,9 +258,8 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
   volatile int* abort_flag = &bars->abort_flag;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n_seg = p.counters[kCtrSegments];
-  const int n_units = n_seg * (p.tiles1 + p.tiles2);
   const int kblocks1 = p.d / kBlockK, kblocks2 = p.I / kBlockK;
+  pdl_launch_dependents();
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
@@ -278,6 +277,10 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
     if (p.split_a) asm volatile("prefetch.tensormap [%0];" ::"l"(&maps1.a2) : "memory");
   }
   if (warp == 1) tmem_alloc(smem_u32(&bars->tmem_base), kTmemCols);
+  // Everything above is independent of the routing result and overlaps the previous kernels.
+  pdl_wait();
+  const int n_seg = p.counters[kCtrSegments];
+  const int n_units = n_seg * (p.tiles1 + p.tiles2);
   tcgen05_fence_before();
   __syncthreads();
   tcgen05_fence_after();
@@ -616,8 +619,7 @@ cudaError_t launch_kernel(const MapSet& m1, const MapSet& m2, const FfnParams& p
                                                  int(Plan<kMaxN>::kSmemBytes));
   if (attr != cudaSuccess) return attr;
   const int grid = min(sm_count(), max_units);
-  ffn_tc_kernel<kMaxN><<<grid, kThreads, Plan<kMaxN>::kSmemBytes, st>>>(m1, m2, p);
-  return cudaGetLastError();
+  return launch_pdl(ffn_tc_kernel<kMaxN>, dim3(grid), dim3(kThreads), Plan<kMaxN>::kSmemBytes, st, 1, m1, m2, p);
 }
 
 }  // namespace

@@ -70,8 +70,10 @@ cudaError_t launch_predict_costs(const void* hidden, const int32_t* ids, const f
 
 // ------------------------------------------------------------------------------------------------
 // Shared pieces of aggregation and selection.
-// Column sum in a fixed order: lane l adds tokens l, l+32, ... in ascending order, then an xor tree.
-// Both the stand-alone and the fused path use this order, so their scores are bit-identical.
+// Column sums D[e] = sum_t costs[t,e] in a fixed order that both the stand-alone and the fused path
+// use, so their scores are bit-identical: with G = blockDim / roundup32(E) groups, group g adds the
+// tokens g, g+G, g+2G, ... in ascending order (thread = expert, so the loads are coalesced), and the
+// G partial sums are added in ascending g.
 // ------------------------------------------------------------------------------------------------
 __device__ __forceinline__ float sortable(float s, int* nonfinite) {
   if (!isfinite(s)) *nonfinite = 1;
@@ -89,25 +91,46 @@ __device__ __forceinline__ int rank_of(const float* s, int E, int e) {
   return r;
 }
 
-__global__ void __launch_bounds__(1024) aggregate_select_kernel(const float* __restrict__ costs, int T, int E, int M,
-                                                                float* __restrict__ scores,
-                                                                int32_t* __restrict__ selected,
-                                                                uint8_t* __restrict__ mask) {
-  __shared__ float s_sc[1024];
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
-  for (int e = warp; e < E; e += nwarp) {
+constexpr int kAggThreads = 512;
+
+// s_part: at least max(kAggThreads, roundup32(E)) floats; s_out: E floats. All threads of the block call.
+__device__ __forceinline__ void aggregate_columns(const float* __restrict__ costs, int T, int E, float* s_part,
+                                                  float* s_out) {
+  const int E_pad = (E + 31) & ~31;
+  const int G = max(1, int(blockDim.x) / E_pad);
+  for (int idx = threadIdx.x; idx < G * E_pad; idx += blockDim.x) {
+    const int g = idx / E_pad, e = idx - g * E_pad;
     float acc = 0.f;
-    for (int t = lane; t < T; t += 32) acc += costs[size_t(t) * E + e];
-    acc = warp_sum(acc);
-    if (lane == 0) {
-      scores[e] = acc;
-      int nf = 0;
-      s_sc[e] = sortable(acc, &nf);
+    if (e < E) {
+#pragma unroll 8
+      for (int t = g; t < T; t += G) acc += costs[size_t(t) * E + e];
     }
+    s_part[idx] = acc;
   }
   __syncthreads();
   for (int e = threadIdx.x; e < E; e += blockDim.x) {
-    const int r = rank_of(s_sc, E, e);
+    float acc = s_part[e];
+    for (int g = 1; g < G; ++g) acc += s_part[g * E_pad + e];
+    s_out[e] = acc;
+  }
+  __syncthreads();
+}
+
+__global__ void __launch_bounds__(kAggThreads) aggregate_select_kernel(const float* __restrict__ costs, int T, int E,
+                                                                     int M, float* __restrict__ scores,
+                                                                     int32_t* __restrict__ selected,
+                                                                     uint8_t* __restrict__ mask) {
+  __shared__ float s_part[1024];
+  __shared__ float s_sc[1024];
+  aggregate_columns(costs, T, E, s_part, s_sc);
+  for (int e = threadIdx.x; e < E; e += blockDim.x) {
+    scores[e] = s_sc[e];
+    int nf = 0;
+    s_part[e] = sortable(s_sc[e], &nf);
+  }
+  __syncthreads();
+  for (int e = threadIdx.x; e < E; e += blockDim.x) {
+    const int r = rank_of(s_part, E, e);
     mask[e] = r < M;
     if (r < M) selected[r] = e;
   }
@@ -115,7 +138,7 @@ __global__ void __launch_bounds__(1024) aggregate_select_kernel(const float* __r
 
 cudaError_t launch_aggregate_select(const float* costs, int T, int E, int M, float* scores, int32_t* sel,
                                     uint8_t* mask, cudaStream_t st) {
-  aggregate_select_kernel<<<1, 1024, 0, st>>>(costs, T, E, M, scores, sel, mask);
+  aggregate_select_kernel<<<1, kAggThreads, 0, st>>>(costs, T, E, M, scores, sel, mask);
   return cudaGetLastError();
 }
 
@@ -156,6 +179,8 @@ __global__ void __launch_bounds__(kGemvWarps * 32) route_scores_kernel(const __n
   __shared__ float s_part[kGemvWarps][16 * 8 + 8];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = lane >> 2, q = lane & 3;
   const int r0 = blockIdx.x * 16, n0 = blockIdx.y * 8;
+  pdl_launch_dependents();
+  pdl_wait();
   auto row_ptr = [&](int r) -> const __nv_bfloat16* {
     r = min(r, 2 * E - 1);
     if (r < E) return (router_w ? router_w : pred_A) + size_t(r) * d;   // router rows unused when logits are given
@@ -223,10 +248,9 @@ cudaError_t launch_route_scores(const void* hidden, const void* router_w, const 
                                 const void* pred_A, float* logits_out, float* raw, float* znorm2, int T, int d,
                                 int E, cudaStream_t st) {
   dim3 grid((2 * E + 15) / 16, (T + 7) / 8);
-  route_scores_kernel<<<grid, kGemvWarps * 32, 0, st>>>(
-      static_cast<const __nv_bfloat16*>(hidden), static_cast<const __nv_bfloat16*>(router_w), router_bias,
-      static_cast<const __nv_bfloat16*>(pred_A), logits_out, raw, znorm2, T, d, E);
-  return cudaGetLastError();
+  return launch_pdl(route_scores_kernel, grid, dim3(kGemvWarps * 32), 0, st, 1,
+                    static_cast<const __nv_bfloat16*>(hidden), static_cast<const __nv_bfloat16*>(router_w), router_bias,
+                    static_cast<const __nv_bfloat16*>(pred_A), logits_out, raw, znorm2, T, d, E);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -248,7 +272,7 @@ cudaError_t launch_route_scores(const void* hidden, const void* router_w, const 
 // ------------------------------------------------------------------------------------------------
 constexpr int kNone = INT_MAX;
 constexpr int kClusterCtas = 8;
-constexpr int kRoutingThreads = 512;
+constexpr int kRoutingThreads = kAggThreads;
 constexpr int kRoutingWarps = kRoutingThreads / 32;
 
 // Order-preserving map float -> uint32 (larger float <=> larger key). Key 0 is never produced by a
@@ -306,9 +330,11 @@ __device__ __forceinline__ uint32_t cluster_cta_rank() {
 template <int NV>
 __global__ void __launch_bounds__(kRoutingThreads) routing_kernel(RoutingArgs a) {
   const int T = a.T, E = a.E, K = a.K, S = T * K;
-  extern __shared__ int32_t s_pos[];   // [S] position of every executed pair inside its expert
+  extern __shared__ int32_t s_dyn[];   // [S] executed routes, then [chunks][E] per-expert token ballots
+  int32_t* s_eids = s_dyn;
+  uint32_t* s_bal = reinterpret_cast<uint32_t*>(s_dyn + S);
+  __shared__ float s_part[kMaxE], s_raw[kMaxE];
   __shared__ float s_sc[kMaxE];
-  __shared__ int32_t s_cnt[kMaxE];
   __shared__ int32_t s_off[kMaxE + 1];
   __shared__ uint8_t s_mask[kMaxE];
   __shared__ int32_t s_wsum[kRoutingWarps], s_wseg[kRoutingWarps];
@@ -321,6 +347,8 @@ __global__ void __launch_bounds__(kRoutingThreads) routing_kernel(RoutingArgs a)
   const int gthread = cta * kRoutingThreads + threadIdx.x;
   constexpr int kAllThreads = kClusterCtas * kRoutingThreads;
   if (threadIdx.x == 0) s_status = 0;
+  pdl_launch_dependents();
+  pdl_wait();
   RT_STAMP(0)
 
   // ---- 1: original routes and predicted costs (one warp per token; a lane owns entries lane+32i)
@@ -396,37 +424,17 @@ __global__ void __launch_bounds__(kRoutingThreads) routing_kernel(RoutingArgs a)
   cluster_barrier();
   RT_STAMP(2)
 
-  // ---- 2: batch aggregation in a fixed order (lane l adds tokens l, l+32, ... ascending, then an
-  // xor tree: the order of aggregate_select_kernel). Every CTA sums all experts itself (the costs are
-  // a few KB in L2), eight experts per warp at a time so that their loads are in flight together.
-  for (int e0 = warp; e0 < E; e0 += kRoutingWarps * 8) {
-    float acc[8];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) acc[j] = 0.f;
-#pragma unroll 2
-    for (int t = lane; t < T; t += 32) {
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        const int e = e0 + j * kRoutingWarps;
-        if (e < E) acc[j] += a.ws.costs[size_t(t) * E + e];
-      }
-    }
-#pragma unroll
-    for (int j = 0; j < 8; ++j) acc[j] = warp_sum(acc[j]);
-    if (lane == 0) {
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        const int e = e0 + j * kRoutingWarps;
-        if (e < E) {
-          int nf = 0;
-          s_sc[e] = sortable(acc[j], &nf);
-          if (nf) atomicOr(&s_status, BASE_DEV_NONFINITE_SCORE);
-          if (cta == 0) {
-            a.ws.scores[e] = acc[j];
-            if (a.dbg.scores) a.dbg.scores[e] = acc[j];
-          }
-        }
-      }
+  // ---- 2: batch aggregation in the fixed order of aggregate_columns(). Every CTA sums all experts
+  // itself (the costs are a few KB in L2): one cluster barrier less than sharing the work.
+  aggregate_columns(a.ws.costs, T, E, s_part, s_raw);
+  for (int e = threadIdx.x; e < E; e += kRoutingThreads) {
+    const float acc = s_raw[e];
+    int nf = 0;
+    s_sc[e] = sortable(acc, &nf);
+    if (nf) atomicOr(&s_status, BASE_DEV_NONFINITE_SCORE);
+    if (cta == 0) {
+      a.ws.scores[e] = acc;
+      if (a.dbg.scores) a.dbg.scores[e] = acc;
     }
   }
 #ifndef BASE_ROUTING_TIMING
@@ -465,46 +473,70 @@ __global__ void __launch_bounds__(kRoutingThreads) routing_kernel(RoutingArgs a)
       }
     }
   }
-  for (int e = threadIdx.x; e < E; e += kRoutingThreads) s_cnt[e] = 0;
+  for (int i = threadIdx.x; i < ((T + 31) >> 5) * E; i += kRoutingThreads) s_bal[i] = 0u;
   __syncthreads();
   RT_STAMP(4)
 
-  // ---- ... and the restricted routes of this CTA's tokens
+  // ---- ... and the restricted routes of this CTA's tokens. Original routes that are still active
+  // keep their place; only the lost ones are replaced, by the best active experts ranked below the
+  // original top-K (every such expert ranks below every original route, so the executed list stays
+  // in router-rank order). Lane k holds the k-th original route.
   for (int t = gwarp; t < T; t += kWarps) {
     uint32_t key[NV], avail = 0;
     const float m = a.ws.tok_m[t], S_t = a.ws.tok_S[t];
+    const int oid = (lane < K) ? a.ws.topk_ids[t * K + lane] : -1;
+    float lv[NV];
+#pragma unroll
+    for (int i = 0; i < NV; ++i) {
+      const int e = lane + 32 * i;
+      lv[i] = (e < E) ? a.logits[size_t(t) * E + e] : -INFINITY;
+    }
+    const float ol = (oid >= 0) ? a.logits[size_t(t) * E + oid] : -INFINITY;
+    const uint32_t okey = float_key(isnan(ol) ? -INFINITY : ol);
+    const bool keep = oid >= 0 && s_mask[oid] != 0;
+    const uint32_t keep_bal = __ballot_sync(0xffffffffu, keep);
+    const int n_keep = __popc(keep_bal);
+    // the last original route bounds the backfill candidates from above
+    const int n_orig = __popc(__ballot_sync(0xffffffffu, oid >= 0));
+    const uint32_t kth_key = __shfl_sync(0xffffffffu, okey, max(n_orig - 1, 0));
+    const int kth_id = __shfl_sync(0xffffffffu, oid, max(n_orig - 1, 0));
 #pragma unroll
     for (int i = 0; i < NV; ++i) {
       const int e = lane + 32 * i;
       key[i] = 0;
       if (e < E) {
-        const float lv = a.logits[size_t(t) * E + e];
-        key[i] = float_key(isnan(lv) ? -INFINITY : lv);
-        bool ok = s_mask[e] != 0;
-        if (ok && a.fill_rule == BASE_FILL_DROP) {
-          ok = false;
-          for (int k = 0; k < K; ++k) ok |= (a.ws.topk_ids[t * K + k] == e);
-        }
-        if (ok) avail |= 1u << i;
+        key[i] = float_key(isnan(lv[i]) ? -INFINITY : lv[i]);
+        const bool below = n_orig == 0 || key[i] < kth_key || (key[i] == kth_key && e > kth_id);
+        if (s_mask[e] != 0 && below && a.fill_rule == BASE_FILL_BACKFILL) avail |= 1u << i;
       }
     }
-    float myq = 0.f;
-    int myid = kNone;
-    for (int k = 0; k < K; ++k) {
+    int myid = keep ? oid : kNone;
+    float myq = keep ? expf(key_float(okey) - m) : 0.f;
+    int mypos = keep ? __popc(keep_bal & ((1u << lane) - 1u)) : -1;
+    const int n_fill = K - n_keep;   // the loop ends early when the active set has no candidate left
+    for (int j = 0; j < n_fill; ++j) {
       uint32_t gk;
       int gi;
       take_best<NV>(key, avail, lane, gk, gi);
-      if (lane == k) {
+      if (gi == kNone) break;
+      // park the j-th backfill in a lane that lost its route (the j-th such lane)
+      const uint32_t lost_bal = ~keep_bal & ((K >= 32) ? 0xffffffffu : ((1u << K) - 1u));
+      const int dst = __fns(lost_bal, 0, j + 1);
+      if (lane == dst) {
         myid = gi;
-        myq = (gi != kNone) ? expf(key_float(gk) - m) : 0.f;
+        myq = expf(key_float(gk) - m);
+        mypos = n_keep + j;
       }
     }
     const float sumq = warp_sum(myq);
     if (lane < K) {
+      // empty slots (budget below K) fill the tail in lane order
+      const uint32_t filled = __ballot_sync((K >= 32) ? 0xffffffffu : ((1u << K) - 1u), mypos >= 0);
+      if (mypos < 0) mypos = __popc(filled) + __popc(~filled & ((1u << lane) - 1u));
       const float den = (a.gate_rule == BASE_GATE_RENORM) ? sumq : S_t;
       const bool ok = myid != kNone;
       const float g = (ok && den > 0.f) ? myq / den : 0.f;
-      const int idx = t * K + lane;
+      const int idx = t * K + mypos;
       a.ws.exec_ids[idx] = ok ? myid : -1;
       a.ws.exec_gates[idx] = g;
       if (a.dbg.exec_ids) a.dbg.exec_ids[idx] = ok ? myid : -1;
@@ -515,35 +547,27 @@ __global__ void __launch_bounds__(kRoutingThreads) routing_kernel(RoutingArgs a)
   cluster_barrier();
   RT_STAMP(6)
 
-  // ---- 4: dispatch lists, computed by every CTA. A warp owns the experts e = warp (mod 16); a lane
-  // holds one token's executed routes in registers. Position of a pair inside its expert = number of
-  // lower-numbered tokens routed to that expert, so each expert's rows are in token order.
-  for (int t0 = 0; t0 < T; t0 += 32) {
-    const int t = t0 + lane;
-    int ids[kMaxK];
-#pragma unroll
-    for (int k = 0; k < kMaxK; ++k) ids[k] = (t < T && k < K) ? a.ws.exec_ids[t * K + k] : -1;
-    for (int e = warp; e < E; e += kRoutingWarps) {
-      int kk = -1;
-#pragma unroll
-      for (int k = 0; k < kMaxK; ++k)
-        if (ids[k] == e) kk = k;
-      const uint32_t bal = __ballot_sync(0xffffffffu, kk >= 0);
-      if (bal) {
-        const int base_cnt = s_cnt[e];
-        if (kk >= 0) s_pos[t * K + kk] = base_cnt + __popc(bal & ((1u << lane) - 1u));
-        __syncwarp();
-        if (lane == 0) s_cnt[e] = base_cnt + __popc(bal);
-      }
+  // ---- 4: dispatch lists, computed by every CTA from a shared-memory copy of the executed routes.
+  // s_bal[chunk][e] is a bitmap of the tokens of a 32-token chunk that go to expert e (set with
+  // shared-memory atomics, so the result does not depend on thread order); positions and counts are
+  // popcounts of these bitmaps, so each expert's rows are in token order.
+  const int n_chunks = (T + 31) >> 5;
+  for (int i = threadIdx.x; i < S; i += kRoutingThreads) {
+    const int e = a.ws.exec_ids[i];
+    s_eids[i] = e;
+    if (e >= 0) {
+      const int t = i / K;
+      atomicOr(&s_bal[(t >> 5) * E + e], 1u << (t & 31));
     }
-    __syncwarp();
   }
   __syncthreads();
   RT_STAMP(7)
   // exclusive scan of the counts (and of the per-expert segment counts) over the block
   {
     const int e = threadIdx.x;   // E <= kRoutingThreads
-    const int c = (e < E) ? s_cnt[e] : 0;
+    int c = 0;
+    if (e < E)
+      for (int ch = 0; ch < n_chunks; ++ch) c += __popc(s_bal[ch * E + e]);
     const int segs = (c + kSegTokens - 1) / kSegTokens;
     int incl = c, sincl = segs;
 #pragma unroll
@@ -599,32 +623,35 @@ __global__ void __launch_bounds__(kRoutingThreads) routing_kernel(RoutingArgs a)
   if (cta == 0)
     for (int i = threadIdx.x; i < a.max_segs; i += kRoutingThreads) a.ws.counters[kCtrReady + i] = 0;
   for (int i = gthread; i < S; i += kAllThreads) {
-    const int e = a.ws.exec_ids[i];
+    const int e = s_eids[i];
     int slot = -1;
     if (e >= 0) {
-      slot = s_off[e] + s_pos[i];
-      a.ws.slot_token[slot] = i / K;
+      const int t = i / K, ch = t >> 5;
+      int pos = __popc(s_bal[ch * E + e] & ((1u << (t & 31)) - 1u));
+      for (int c2 = 0; c2 < ch; ++c2) pos += __popc(s_bal[c2 * E + e]);
+      slot = s_off[e] + pos;
+      a.ws.slot_token[slot] = t;
     }
     a.ws.token_slot[i] = slot;
   }
   RT_STAMP(9)
 }
 
-constexpr size_t kRoutingMaxSmem = size_t(kMaxSlots) * 4;
+constexpr size_t kRoutingMaxSmem = size_t(kMaxSlots) * 4 + size_t(kMaxT / 32) * kMaxE * 4;
 
 template <int NV>
 cudaError_t launch_routing_nv(const RoutingArgs& a, cudaLaunchConfig_t* cfg) {
   static cudaError_t attr = cudaFuncSetAttribute(routing_kernel<NV>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                  int(kRoutingMaxSmem));
   if (attr != cudaSuccess) return attr;
-  return cudaLaunchKernelEx(cfg, routing_kernel<NV>, a);
+  return launch_pdl(routing_kernel<NV>, cfg->gridDim, cfg->blockDim, cfg->dynamicSmemBytes, cfg->stream, kClusterCtas, a);
 }
 
 cudaError_t launch_routing(const RoutingArgs& a, cudaStream_t st) {
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3(kClusterCtas);
   cfg.blockDim = dim3(kRoutingThreads);
-  cfg.dynamicSmemBytes = size_t(a.T) * a.K * 4;
+  cfg.dynamicSmemBytes = size_t(a.T) * a.K * 4 + size_t((a.T + 31) / 32) * a.E * 4;
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -650,6 +677,8 @@ __global__ void __launch_bounds__(256) gather_kernel(const __nv_bfloat16* __rest
                                                      const int32_t* __restrict__ counters,
                                                      __nv_bfloat16* __restrict__ x_sorted, int d) {
   const int slot = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  pdl_launch_dependents();
+  pdl_wait();
   if (slot >= counters[kCtrSlots]) return;
   const int t = slot_token[slot];
   const uint4* src = reinterpret_cast<const uint4*>(hidden + size_t(t) * d);
@@ -671,9 +700,8 @@ __global__ void __launch_bounds__(256) gather_kernel(const __nv_bfloat16* __rest
 }
 
 cudaError_t launch_gather(const void* hidden, const Workspace& ws, int T, int K, int d, cudaStream_t st) {
-  gather_kernel<<<(T * K + 7) / 8, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(hidden), ws.slot_token, ws.counters,
-                                                 ws.x_sorted, d);
-  return cudaGetLastError();
+  return launch_pdl(gather_kernel, dim3((T * K + 7) / 8), dim3(256), 0, st, 1,
+                    static_cast<const __nv_bfloat16*>(hidden), ws.slot_token, ws.counters, ws.x_sorted, d);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -694,6 +722,8 @@ __global__ void __launch_bounds__(256) combine_kernel(const float* __restrict__ 
   __shared__ int s_slot[kMaxK];
   __shared__ float s_gate[kMaxK];
   __shared__ float s_red[8];
+  pdl_launch_dependents();
+  pdl_wait();
   if (threadIdx.x < kMaxK) {
     const bool in = threadIdx.x < K;
     s_slot[threadIdx.x] = in ? token_slot[t * K + threadIdx.x] : -1;
@@ -767,10 +797,9 @@ __global__ void __launch_bounds__(256) combine_kernel(const float* __restrict__ 
 
 cudaError_t launch_combine(const Workspace& ws, const void* hidden, void* out, int out_is_fp32, void* x_next,
                            int T, int K, int d, cudaStream_t st) {
-  combine_kernel<<<T, 256, 0, st>>>(ws.ypair, ws.token_slot, ws.exec_gates,
-                                    static_cast<const __nv_bfloat16*>(hidden), out, out_is_fp32,
-                                    static_cast<__nv_bfloat16*>(x_next), K, d);
-  return cudaGetLastError();
+  return launch_pdl(combine_kernel, dim3(T), dim3(256), 0, st, 1, ws.ypair, ws.token_slot, ws.exec_gates,
+                    static_cast<const __nv_bfloat16*>(hidden), out, out_is_fp32, static_cast<__nv_bfloat16*>(x_next), K,
+                    d);
 }
 
 }  // namespace base
