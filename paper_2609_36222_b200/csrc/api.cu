@@ -1,6 +1,5 @@
 // C-ABI entry points: argument checks, workspace carving, kernel sequencing. No device allocation,
 // no synchronisation (except the *_host entry point, which waits for its own copies).
-#include <stdlib.h>
 #include <string.h>
 
 #include "common.cuh"
@@ -79,21 +78,19 @@ int enqueue_layer(const LayerCall& c, const Workspace& ws, cudaStream_t st, int*
   ra.dbg = c.dbg;
   e = launch_routing(ra, st);
   if (e != cudaSuccess) return cuda_fail(e);
-#ifdef BASE_ROUTING_TIMING
-  if (getenv("BASE_DOUBLE_ROUTING")) launch_routing(ra, st);
-#endif
   ++*launches;
   mark(2, st);
 
-  e = launch_gather(c.hidden, ws, c.T, s.K, s.d, st);
-  if (e != cudaSuccess) return cuda_fail(e);
-  ++*launches;
-
+  if (c.opt.ffn_impl == 1) {
+    e = launch_gather(c.hidden, ws, c.T, s.K, s.d, st);   // the streaming kernel gathers by itself
+    if (e != cudaSuccess) return cuda_fail(e);
+    ++*launches;
+  }
   mark(3, st);
   if (c.opt.ffn_impl == 1) {
     e = launch_ffn_simple(s, *c.w, ws, st, launches);
   } else {
-    e = launch_ffn_tc(s, *c.w, ws, c.T, st, launches);
+    e = launch_ffn_tc(s, *c.w, c.hidden, ws, c.T, st, launches);
   }
   if (e != cudaSuccess) return cuda_fail(e);
   mark(4, st);

@@ -106,7 +106,8 @@ struct Workspace {
   size_t bytes;
 };
 
-constexpr int kCtrDispatched = 0, kCtrSegments = 1, kCtrStatus = 2, kCtrSlots = 3, kCtrTicket = 4, kCtrReady = 16;
+constexpr int kCtrDispatched = 0, kCtrSegments = 1, kCtrStatus = 2, kCtrSlots = 3, kCtrTicket = 4, kCtrGather = 5,
+              kCtrReady = 16;
 constexpr int kRowPad = 256;  // rows readable past the last sorted row (tile over-read stays in bounds)
 
 inline int max_segments(int E, int T, int K) { return E + (T * K) / kSegTokens + 1; }

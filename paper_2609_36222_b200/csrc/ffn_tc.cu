@@ -18,6 +18,13 @@
 // k-blocks land in shared memory already in the layout the MMA descriptors expect; the token box
 // comes from a tensor map whose box height equals the padded token count of the unit.
 //
+// Both passes run in ONE launch. Work units (all gate/up tiles, then all down tiles) are handed out by
+// a global ticket; a down unit waits (bounded) on a per-segment counter of finished gate/up tiles.
+// Because gate/up units never wait and are all taken before any down unit, the scheme cannot
+// deadlock as long as the grid is co-resident (it is: at most one CTA per SM). The gather of the
+// token inputs into expert-sorted order is done by the epilogue warps while the first weight boxes
+// are already in flight.
+//
 // Every wait is bounded: on expiry the CTA raises an abort flag, all roles leave their loops, TMEM
 // is freed and BASE_DEV_WAIT_EXPIRED is OR-ed into the status word.
 #include <cuda.h>
@@ -32,7 +39,6 @@ namespace base {
 namespace {
 
 constexpr int kBlockK = 64;                 // bf16 per k-block = one 128-byte swizzled row
-constexpr int kKbPerStage = 2;              // k-blocks per pipeline stage
 constexpr int kTileABytes = 128 * 128;      // one k-block of the weight tile: 128 rows x 128 B
 constexpr int kThreads = 192;
 constexpr int kMaxStages = 8;
@@ -43,10 +49,13 @@ constexpr long long kWaitCycles = 4000000000ll;   // about 2 s of SM clock
 
 // Shared-memory plan for work units of at most kMaxN tokens: the smaller the token tile, the more
 // weight stages fit.
+constexpr int kb_per_stage(int /*max_n*/) { return 2; }   // k-blocks per pipeline stage (256 B per weight row and box)
+
 template <int kMaxN>
 struct Plan {
+  static constexpr int kKb = kb_per_stage(kMaxN);
   static constexpr int kTileBBytes = kMaxN * 128;                                  // per k-block
-  static constexpr int kStageBytes = kKbPerStage * (kTileABytes + kTileBBytes);
+  static constexpr int kStageBytes = kKb * (kTileABytes + kTileBBytes);
   static constexpr int kExBytes = kMaxN * 64 * 4;   // up-projection exchange buffer [token][row] fp32
   static constexpr int kFixed = 1024 /*alignment slack*/ + 512 /*barriers*/;
   static constexpr int kFit = (kSmemLimit - kFixed - kExBytes) / kStageBytes;
@@ -57,6 +66,14 @@ struct Plan {
   static_assert(kStages >= 2, "need at least two stages");
 };
 
+// Work units of one launch, in execution order: all gate/up tiles (segment-major), then all down
+// tiles. CTA c takes units c, c + grid, c + 2 grid, ...: every CTA finishes its gate/up units before
+// it touches a down unit, so the dependency of a down unit (all gate/up tiles of its segment) is
+// always on work that never waits itself.
+struct Unit {
+  int phase, seg, expert, offset, count, npad, tile;
+};
+
 struct Bars {
   unsigned long long full[kMaxStages];
   unsigned long long empty[kMaxStages];
@@ -64,6 +81,8 @@ struct Bars {
   unsigned long long acc_empty[2];
   uint32_t tmem_base;
   int abort_flag;
+  Unit stage_unit[kMaxStages];  // decoded unit travelling with each stage (phase 0 = no more work)
+  Unit acc_unit[2];             // unit of each accumulator stage
 };
 static_assert(sizeof(Bars) <= 512, "barrier block must fit its reserved space");
 
@@ -82,6 +101,9 @@ struct FfnParams {
   int32_t* counters;
   __nv_bfloat16* h;     // gate/up pass output
   float* ypair;         // down pass output
+  const __nv_bfloat16* hidden;   // [T,d] token inputs
+  __nv_bfloat16* x_sorted;       // [rows,d] token inputs in expert-sorted order (written here)
+  const int32_t* slot_token;     // [rows] token of every sorted row
   int I, d;
   int tiles1, tiles2;   // work units per segment: I/64 gate/up tiles, d/128 down tiles
   int steps1, steps2;   // pipeline stages per unit: ceil(d/64 / 2), ceil(I/64 / 2)
@@ -210,14 +232,6 @@ __device__ __forceinline__ bool named_and(int id, int threads, bool pred) {
   return out != 0;
 }
 
-// Work units of one launch, in execution order: all gate/up tiles (segment-major), then all down
-// tiles. CTA c takes units c, c + grid, c + 2 grid, ...: every CTA finishes its gate/up units before
-// it touches a down unit, so the dependency of a down unit (all gate/up tiles of its segment) is
-// always on work that never waits itself.
-struct Unit {
-  int phase, seg, expert, offset, count, npad, tile;
-};
-
 __device__ __forceinline__ Unit decode_unit(const FfnParams& p, int u, int n_seg) {
   Unit r;
   const int u1 = n_seg * p.tiles1;
@@ -249,12 +263,13 @@ __global__ void __launch_bounds__(kThreads, 1)
 ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapSet maps2, const FfnParams p) {
   using P = Plan<kMaxN>;
   constexpr int kStages = P::kStages, kStageBytes = P::kStageBytes, kAccCols = P::kAccCols, kTmemCols = P::kTmemCols;
+  constexpr int kKbPerStage = P::kKb;
   constexpr int kStageABytes = kKbPerStage * kTileABytes;
   extern __shared__ unsigned char smem_raw[];
   unsigned char* base_ptr = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   unsigned char* stages = base_ptr;
-  float* ex = reinterpret_cast<float*>(base_ptr + size_t(kStages) * kStageBytes);
-  Bars* bars = reinterpret_cast<Bars*>(base_ptr + size_t(kStages) * kStageBytes + P::kExBytes);
+  float* ex = reinterpret_cast<float*>(base_ptr + size_t(P::kStages) * kStageBytes);
+  Bars* bars = reinterpret_cast<Bars*>(base_ptr + size_t(P::kStages) * kStageBytes + P::kExBytes);
   volatile int* abort_flag = &bars->abort_flag;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -267,7 +282,7 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
       mbar_init(smem_u32(&bars->empty[s]), 1);
     }
     for (int a = 0; a < 2; ++a) {
-      mbar_init(smem_u32(&bars->acc_full[a]), 1);
+      mbar_init(smem_u32(&bars->acc_full[a]), 2);     // the MMA completion and the unit id hand-over
       mbar_init(smem_u32(&bars->acc_empty[a]), 128);
     }
     bars->abort_flag = 0;
@@ -281,25 +296,37 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
   pdl_wait();
   const int n_seg = p.counters[kCtrSegments];
   const int n_units = n_seg * (p.tiles1 + p.tiles2);
+  const int n_slots = p.counters[kCtrSlots];
   tcgen05_fence_before();
   __syncthreads();
   tcgen05_fence_after();
   const uint32_t tmem_base = bars->tmem_base;
 
   if (warp == 0) {
-    // ---------------------------------------------------------------- TMA producer
+    // ---------------------------------------------------------------- TMA producer + unit scheduler
+    // Units are handed out by a global ticket, in list order: whoever is free takes the next one, so
+    // all CTAs finish within one (small) unit of each other. The unit id travels with the stage.
     if (lane == 0) {
       int stage = 0;
       uint32_t phase = 0;
-      bool ok = true;
-      for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
-        const Unit un = decode_unit(p, u, n_seg);
+      bool ok = true, x_ready = false;
+      // the ticket and the decoding of the next unit are requested one unit ahead, so their memory
+      // latency never stalls the weight stream
+      int u_cur = atomicAdd(p.counters + kCtrTicket, 1);
+      Unit un_next = decode_unit(p, min(u_cur, max(n_units - 1, 0)), n_seg);
+      while (ok && u_cur < n_units) {
+        const Unit un = un_next;
+        int u_next = n_units;
         const bool gu = un.phase == 1;
         const int arow = gu ? un.expert * p.I + un.tile * 64 : un.expert * p.d + un.tile * 128;
         const CUtensorMap* tm_b = gu ? &maps1.b[(un.npad >> 4) - 1] : &maps2.b[(un.npad >> 4) - 1];
         const uint32_t bytes = uint32_t(kKbPerStage * (kTileABytes + un.npad * 128));
         const int n_steps = gu ? p.steps1 : p.steps2;
-        bool h_ready = gu;   // a down unit reads h rows that other CTAs write
+        // The token operand of a unit is produced by other CTAs: the gathered inputs (gate/up units)
+        // or the h rows of the segment (down units). Weight boxes do not depend on it and go first.
+        bool b_ready = gu ? x_ready : false;
+        const int32_t* flag = gu ? p.counters + kCtrGather : p.counters + kCtrReady + un.seg;
+        const int need = gu ? n_slots : p.tiles1;
         for (int st = 0; st < n_steps; ++st) {
           if (!mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1u, abort_flag)) {
             ok = false;
@@ -309,6 +336,8 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
           const uint32_t full = smem_u32(&bars->full[stage]);
           const uint32_t sa = smem_u32(stages + size_t(stage) * kStageBytes);
           const uint32_t sb = sa + kStageABytes;
+          bars->stage_unit[stage] = un;
+          if (st == 0) u_next = atomicAdd(p.counters + kCtrTicket, 1);
           // k-blocks past the end of K are out of the tensor's bounds and arrive as zeros; the box
           // always delivers its full byte count.
           mbar_expect_tx(full, bytes);
@@ -325,35 +354,38 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
           } else {
             tma_load_3d(sa, &maps2.a, 0, arow, kb, full);            // {elem, row, k-block}
           }
-          if (!h_ready) {
-            // The weight box above is already in flight; now wait (bounded) until every gate/up tile
-            // of this segment has published its h rows.
-            const int32_t* flag = p.counters + kCtrReady + un.seg;
+          if (!b_ready) {
             const long long t0 = clock64();
-            bool ready = false;
 #pragma unroll 1
             for (uint32_t it = 0; it < kSpinLimit; ++it) {
-              if (ld_acquire(flag) >= p.tiles1) {
-                ready = true;
+              if (ld_acquire(flag) >= need) {
+                b_ready = true;
                 break;
               }
               __nanosleep(64);
               if ((it & 255u) == 255u && (*abort_flag || clock64() - t0 > kWaitCycles)) break;
             }
-            if (!ready) {
+            if (!b_ready) {
               *abort_flag = 1;
               ok = false;
               break;
             }
             asm volatile("fence.proxy.async;" ::: "memory");   // generic-proxy writes -> async-proxy (TMA) reads
-            h_ready = true;
+            if (gu) x_ready = true;
           }
           tma_load_3d(sb, tm_b, 0, un.offset, kb, full);
           if (++stage == kStages) {
             stage = 0;
             phase ^= 1u;
           }
+          if (st == 0 && u_next < n_units) un_next = decode_unit(p, u_next, n_seg);
         }
+        u_cur = u_next;
+      }
+      // end of work: one more stage that carries the stop mark
+      if (ok && mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1u, abort_flag)) {
+        bars->stage_unit[stage].phase = 0;
+        mbar_arrive(smem_u32(&bars->full[stage]));
       }
     }
     __syncwarp();
@@ -362,18 +394,25 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
     if (lane == 0) {
       int stage = 0, acc = 0;
       uint32_t phase = 0, acc_phase = 0;
-      bool ok = true;
-      for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
-        const Unit un = decode_unit(p, u, n_seg);
+      while (true) {
+        if (!mbar_wait(smem_u32(&bars->full[stage]), phase, abort_flag)) break;
+        const Unit un = bars->stage_unit[stage];
+        if (!mbar_wait(smem_u32(&bars->acc_empty[acc]), acc_phase ^ 1u, abort_flag)) break;
+        bars->acc_unit[acc] = un;
+        if (un.phase == 0) {
+          // pass the stop mark on to the epilogue (both arrivals of the barrier)
+          mbar_arrive(smem_u32(&bars->acc_full[acc]));
+          mbar_arrive(smem_u32(&bars->acc_full[acc]));
+          break;
+        }
         const int n_steps = un.phase == 1 ? p.steps1 : p.steps2;
         const int kblocks = un.phase == 1 ? kblocks1 : kblocks2;
-        if (!mbar_wait(smem_u32(&bars->acc_empty[acc]), acc_phase ^ 1u, abort_flag)) break;
-        tcgen05_fence_after();
         const uint32_t d_tmem = tmem_base + uint32_t(acc * kAccCols);
         const uint32_t idesc = make_idesc(un.npad);
         const uint32_t tile_b = uint32_t(un.npad * 128);
+        bool ok = true;
         for (int st = 0; st < n_steps; ++st) {
-          if (!mbar_wait(smem_u32(&bars->full[stage]), phase, abort_flag)) {
+          if (st > 0 && !mbar_wait(smem_u32(&bars->full[stage]), phase, abort_flag)) {
             ok = false;
             break;
           }
@@ -398,22 +437,52 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
         }
         if (!ok) break;
         umma_commit(smem_u32(&bars->acc_full[acc]));
+        mbar_arrive(smem_u32(&bars->acc_full[acc]));   // releases acc_unit[acc] to the epilogue
         acc ^= 1;
         if (acc == 0) acc_phase ^= 1u;
       }
     }
     __syncwarp();
   } else {
-    // ---------------------------------------------------------------- epilogue warps (TMEM -> global)
+    // ---------------------------------------------------------------- epilogue warps
     const int q = warp & 3;  // TMEM lane quarter this warp may read
+    // First job: gather the token inputs into expert-sorted order (x_sorted[row] = hidden[token of
+    // row]), rows dealt round-robin over all CTAs. The weight stream is already running; only the
+    // first token box of a gate/up unit waits for the global row count.
+    {
+      const int ew = warp - 2;
+      const int dv = p.d >> 3;
+      for (int row = blockIdx.x * 4 + ew; row < n_slots; row += gridDim.x * 4) {
+        const int t = p.slot_token[row];
+        const uint4* src = reinterpret_cast<const uint4*>(p.hidden + size_t(t) * p.d);
+        uint4* dst = reinterpret_cast<uint4*>(p.x_sorted + size_t(row) * p.d);
+        for (int j0 = 0; j0 < dv; j0 += 256) {
+          uint4 v[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const int j = j0 + i * 32 + lane;
+            if (j < dv) v[i] = __ldg(src + j);
+          }
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const int j = j0 + i * 32 + lane;
+            if (j < dv) dst[j] = v[i];
+          }
+        }
+        __threadfence();
+        __syncwarp();
+        if (lane == 0) red_release_add(p.counters + kCtrGather, 1);
+      }
+    }
     int acc = 0;
     uint32_t acc_phase = 0;
-    for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
-      const Unit un = decode_unit(p, u, n_seg);
+    while (true) {
       int got = 0;
       if (lane == 0) got = mbar_wait(smem_u32(&bars->acc_full[acc]), acc_phase, abort_flag, 128) ? 1 : 0;
       got = __shfl_sync(0xffffffffu, got, 0);
       if (!named_and(1, 128, got != 0)) break;
+      const Unit un = bars->acc_unit[acc];
+      if (un.phase == 0) break;
       tcgen05_fence_after();
       const uint32_t taddr = tmem_base + (uint32_t(q * 32) << 16) + uint32_t(acc * kAccCols);
       if (un.phase == 1) {
@@ -581,7 +650,7 @@ bool map_rows_kblocks(const void* ptr, uint64_t rows, uint64_t cols, uint32_t bo
 // Gate and up matrices seen through one map {64 elements, rows, {gate, up}, k-blocks}: the third
 // coordinate steps from W_gate to W_up, which works whenever W_up lies above W_gate at a distance
 // the tensor map can express.
-bool map_gate_up(const void* gate, const void* up, uint64_t rows, uint64_t cols, CUtensorMap* out) {
+bool map_gate_up(const void* gate, const void* up, uint64_t rows, uint64_t cols, uint32_t box_kb, CUtensorMap* out) {
   const uintptr_t g = reinterpret_cast<uintptr_t>(gate), u = reinterpret_cast<uintptr_t>(up);
   if (u <= g) return false;
   const uint64_t delta = u - g;
@@ -599,7 +668,7 @@ bool map_gate_up(const void* gate, const void* up, uint64_t rows, uint64_t cols,
   k.box[0] = kBlockK;
   k.box[1] = 64;
   k.box[2] = 2;
-  k.box[3] = kKbPerStage;
+  k.box[3] = box_kb;
   return encode_map(k, out);
 }
 
@@ -624,13 +693,15 @@ cudaError_t launch_kernel(const MapSet& m1, const MapSet& m2, const FfnParams& p
 
 }  // namespace
 
-cudaError_t launch_ffn_tc(const base_layer_shape& s, const base_layer_weights& w, const Workspace& ws, int T,
-                          cudaStream_t st, int* launches) {
+cudaError_t launch_ffn_tc(const base_layer_shape& s, const base_layer_weights& w, const void* hidden,
+                          const Workspace& ws, int T, cudaStream_t st, int* launches) {
   const uint64_t slots = uint64_t(T) * s.K + kRowPad;
   const uint64_t wrows = uint64_t(s.E) * s.I;
   MapSet m1{}, m2{};
   FfnParams p{};
-  if (map_gate_up(w.w_gate, w.w_up, wrows, s.d, &m1.a)) {
+  const int max_n = T <= 32 ? 32 : (T <= 64 ? 64 : 128);
+  const uint32_t kKbPerStage = uint32_t(kb_per_stage(max_n));
+  if (map_gate_up(w.w_gate, w.w_up, wrows, s.d, kKbPerStage, &m1.a)) {
     p.split_a = 0;
   } else {
     p.split_a = 1;
@@ -651,12 +722,15 @@ cudaError_t launch_ffn_tc(const base_layer_shape& s, const base_layer_weights& w
   p.counters = ws.counters;
   p.h = ws.h;
   p.ypair = ws.ypair;
+  p.hidden = static_cast<const __nv_bfloat16*>(hidden);
+  p.x_sorted = ws.x_sorted;
+  p.slot_token = ws.slot_token;
   p.I = s.I;
   p.d = s.d;
   p.tiles1 = s.I / 64;
   p.tiles2 = s.d / 128;
-  p.steps1 = (s.d / kBlockK + kKbPerStage - 1) / kKbPerStage;
-  p.steps2 = (s.I / kBlockK + kKbPerStage - 1) / kKbPerStage;
+  p.steps1 = (s.d / kBlockK + int(kKbPerStage) - 1) / int(kKbPerStage);
+  p.steps2 = (s.I / kBlockK + int(kKbPerStage) - 1) / int(kKbPerStage);
   const int max_units = segs * (p.tiles1 + p.tiles2);
   // No expert can receive more tokens than the batch holds, which bounds the token tile.
   cudaError_t e;

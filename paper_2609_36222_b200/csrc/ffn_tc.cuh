@@ -3,6 +3,6 @@
 #include "common.cuh"
 
 namespace base {
-cudaError_t launch_ffn_tc(const base_layer_shape& s, const base_layer_weights& w, const Workspace& ws, int T,
-                          cudaStream_t st, int* launches);
+cudaError_t launch_ffn_tc(const base_layer_shape& s, const base_layer_weights& w, const void* hidden,
+                          const Workspace& ws, int T, cudaStream_t st, int* launches);
 }

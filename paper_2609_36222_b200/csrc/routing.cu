@@ -614,6 +614,7 @@ __global__ void __launch_bounds__(kRoutingThreads) routing_kernel(RoutingArgs a)
       a.ws.counters[kCtrSlots] = off + c;
       a.ws.counters[kCtrStatus] = s_status;
       a.ws.counters[kCtrTicket] = 0;
+      a.ws.counters[kCtrGather] = 0;
       if (a.dbg.n_dispatched) a.dbg.n_dispatched[0] = ndisp;
       if (a.dbg.status) a.dbg.status[0] = s_status;
     }
