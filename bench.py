@@ -30,6 +30,9 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
 NOMINAL_HBM_GBS = 8000.0
+# DRAM bytes (read + written) of one FFN launch from the committed ncu capture of the same workload
+# (profiles/ffn_tc_kernel_qwen3_b64_m32.md); other workloads have no capture and report null.
+NCU_FFN_TRAFFIC = {("qwen3", 64, 32): 303.55e6 + 7.83e6}
 FALLBACK_HBM_GBS = 6650.0
 
 
@@ -185,17 +188,13 @@ def run_ours(args, cfg, T, M):
     from paper_2609_36222_b200 import workloads as wl
     from paper_2609_36222_b200.layer import DeviceLayer, bits_to_device
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    from paper_2609_36222_b200 import multi
+    rank, world, local = multi.env_ranks()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the CUDA path has no CPU fallback")
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=dev)
+    dist = multi.init_process_group("nccl", dev)
 
     peaks, peak_kind = measured_peaks()
     hbm_peak = float(peaks.get("hbm_gbs", FALLBACK_HBM_GBS))
@@ -210,9 +209,10 @@ def run_ours(args, cfg, T, M):
             n_rep = max(2, int(40e9 // (cfg.E * cfg.expert_bytes)))
     shape = (cfg.d, cfg.E, cfg.K, cfg.I)
     ws = B.alloc_workspace(max(B.layer_workspace_bytes(*shape, T), B.stack_workspace_bytes(*shape, T)), dev)
-    base_layer = rank * 1000
-    layers = [DeviceLayer(cfg, dev, layer=base_layer + r, T_max=T, workspace=ws) for r in range(n_rep)]
-    hidden = [bits_to_device(wl.hidden_bits(cfg, T, layer=base_layer + r), dev) for r in range(n_rep)]
+    layer_ids = multi.replica_layer_ids(rank, n_rep)
+    base_layer = layer_ids[0]
+    layers = [DeviceLayer(cfg, dev, layer=l, T_max=T, workspace=ws) for l in layer_ids]
+    hidden = [bits_to_device(wl.hidden_bits(cfg, T, layer=l), dev) for l in layer_ids]
     out = torch.empty(T, cfg.d, dtype=torch.bfloat16, device=dev)
     nd_buf = torch.zeros(max(n_rep, 1), dtype=torch.int32, device=dev)
     stream = torch.cuda.Stream(device=dev)
@@ -275,10 +275,7 @@ def run_ours(args, cfg, T, M):
         if ms * args.steps < 300 and not args.profile:
             timed(graphs, max(args.steps, int(300 / max(ms, 1e-3))), 0)
     clk = clocks.summary()
-    if dist is not None:
-        t = torch.tensor([ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = multi.max_over_ranks(ms, dist, dev)
 
     # ---- per-kernel pass for the roofline: the library records the caller's events around the FFN kernels
     n_prof = min(args.steps, 40)
@@ -328,11 +325,8 @@ def run_ours(args, cfg, T, M):
             B.base_moe_decode_layer_host(shape, layers[r].weights, h_in[r], M, h_out, hws, h_n_dispatched=h_nd,
                                          stream=stream)
         e2e_us = (time.perf_counter() - t0) / args.steps * 1e6
-        if dist is not None:
-            t = torch.tensor([e2e_us], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_us = float(t.item())
-        e2e = {"value": e2e_us / world, "unit": "us/step", "h2d_bytes_per_step": T * cfg.d * 2,
+        e2e_us = multi.max_over_ranks(e2e_us, dist, dev)
+        e2e = {"value": multi.whole_job_us_per_step(e2e_us / 1e3, world), "unit": "us/step", "h2d_bytes_per_step": T * cfg.d * 2,
                "d2h_bytes_per_step": T * cfg.d * 2 + 4}
 
     if rank != 0:
@@ -345,7 +339,8 @@ def run_ours(args, cfg, T, M):
     step_bytes = algorithmic_bytes(cfg, T, mean_nd)
     gbs = step_bytes / (per_layer_us * 1e-6) / 1e9
     line = {
-        "metric": "moe_decode_layer_us_per_step", "value": us / world, "unit": "us/step", "n_gpus": world,
+        "metric": "moe_decode_layer_us_per_step", "value": multi.whole_job_us_per_step(ms, world), "unit": "us/step",
+        "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": False,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {
@@ -370,7 +365,8 @@ def run_ours(args, cfg, T, M):
         fb = ffn_algorithmic_bytes(cfg, T, mean_nd)
         ach = fb / (ffn_us * 1e-6) / 1e9
         line["roofline"] = {"bound": "hbm", "kernel": "grouped SwiGLU FFN (gate/up + down)", "achieved": ach,
-                            "peak": hbm_peak, "unit": "GB/s", "frac": ach / hbm_peak, "traffic": None,
+                            "peak": hbm_peak, "unit": "GB/s", "frac": ach / hbm_peak,
+                            "traffic": NCU_FFN_TRAFFIC.get((cfg.name, T, M)),
                             "us_per_launch": ffn_us, "peak_kind": f"of {peak_kind}",
                             "algorithmic_bytes_per_launch": fb}
         line["kernel_us"] = stage_us

@@ -1,0 +1,56 @@
+"""Multi-GPU plumbing of the benchmark: one process per GPU, independent decode batches per rank.
+
+The method has no exchange step between decode batches (the active set is chosen per batch), so
+N GPUs run N independent replicas of the layer ("replicas only", weak scaling). The only
+communication is the timing protocol: a barrier on both sides of the timed region and the
+maximum of the per-rank times.
+"""
+
+from __future__ import annotations
+
+import os
+
+
+def env_ranks():
+    """(rank, world_size, local_rank) from the torchrun environment (1 process when absent)."""
+    return (int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1")),
+            int(os.environ.get("LOCAL_RANK", "0")))
+
+
+def init_process_group(backend: str, device=None):
+    """Join the job when WORLD_SIZE > 1; returns the torch.distributed module or None."""
+    rank, world, _ = env_ranks()
+    if world <= 1:
+        return None
+    import torch.distributed as dist
+    if not dist.is_initialized():
+        kw = {"device_id": device} if (backend == "nccl" and device is not None) else {}
+        dist.init_process_group(backend, **kw)
+    return dist
+
+
+def replica_layer_ids(rank: int, n_replicas: int, per_rank_stride: int = 1000):
+    """Seeded layer ids of the weight replicas a rank rotates through; disjoint across ranks."""
+    assert n_replicas <= per_rank_stride
+    return [rank * per_rank_stride + r for r in range(n_replicas)]
+
+
+def max_over_ranks(value: float, dist, device="cpu") -> float:
+    """Slowest rank's value (all ranks receive it)."""
+    if dist is None:
+        return float(value)
+    import torch
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def barrier(dist):
+    if dist is not None:
+        dist.barrier()
+
+
+def whole_job_us_per_step(ms_per_step_max: float, world: int) -> float:
+    """Whole-job figure of the time-like metric: the job completes `world` layer steps (one per
+    rank) in the slowest rank's step time."""
+    return ms_per_step_max * 1e3 / max(world, 1)
