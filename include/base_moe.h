@@ -41,7 +41,8 @@ enum {
   BASE_ERR_INVALID_ARG = 1,        /* null / misaligned pointer, non-positive size, bad enum */
   BASE_ERR_UNSUPPORTED = 2,        /* shape outside the compiled limits (see each call) */
   BASE_ERR_WORKSPACE_TOO_SMALL = 3,
-  BASE_ERR_CUDA = 4                /* a CUDA call failed; base_last_cuda_error() has the code */
+  BASE_ERR_CUDA = 4,               /* a CUDA call failed; base_last_cuda_error() has the code */
+  BASE_ERR_SCRATCH_LIMIT = 5       /* base_moe_decode_layer_noalloc: the shape needs more scratch than the built-in buffer */
 };
 
 enum {                             /* bits of the device status word */
@@ -148,6 +149,38 @@ int base_moe_decode_layer(const base_layer_shape* shape, const base_layer_weight
                           const uint8_t* forced_mask, void* out, const base_layer_options* opt,
                           const base_layer_debug* dbg, void* workspace, size_t workspace_bytes,
                           void* stream);
+
+/*
+ * The paper has no counterpart to this entry point; it exists for callers that must not allocate.
+ *
+ * base_moe_decode_layer needs a scratch workspace that somebody has to cudaMalloc. Some callers cannot
+ * do that at the moment they need the layer: a plug-in that runs inside another engine's decode loop
+ * after that engine has handed every free byte of the GPU to its KV cache; a component that is only
+ * given a stream and tensors, not an allocator; a latency-critical loop whose owner forbids calls that
+ * may synchronise the device or fail for lack of memory. For them this variant does
+ * the same decode step with the same arguments minus the workspace: its scratch is a fixed buffer of
+ * BASE_NOALLOC_SCRATCH_BYTES (16 MiB) that is part of the library image. Every GPU that loads the
+ * library carries that buffer until the process exits, whether the entry point is used or not.
+ *
+ *  - Shapes whose workspace (base_moe_decode_layer_workspace_bytes) exceeds the buffer are refused with
+ *    BASE_ERR_SCRATCH_LIMIT and nothing is enqueued. 16 MiB covers, for example, the Qwen3-30B-A3B
+ *    shape (d 2048, E 128, K 8, I 768) up to 128 tokens.
+ *  - The call allocates no device memory and frees none (no cudaMalloc/cudaFree, no allocating library
+ *    routine); it only enqueues kernels on `stream`.
+ *  - The first call on each device looks up the buffer's device address (cudaGetSymbolAddress, with
+ *    that device current). Make that first call outside any stream capture.
+ *  - All calls on a device share the one buffer, and it keeps whatever the previous call left in it.
+ *    The layer re-initialises the few counters it needs to start from zero by itself, so back-to-back
+ *    calls on one stream are fine; two calls that overlap on the GPU (different streams, or graphs
+ *    replayed concurrently) race on the buffer and give wrong results. The same holds between this
+ *    entry point and nothing else: base_moe_decode_layer never touches the built-in buffer.
+ * Arguments, limits, options and debug outputs are those of base_moe_decode_layer.
+ */
+#define BASE_NOALLOC_SCRATCH_BYTES (16u << 20)
+int base_moe_decode_layer_noalloc(const base_layer_shape* shape, const base_layer_weights* weights,
+                                  const void* hidden_bf16, const float* router_logits, int T, int budget,
+                                  const uint8_t* forced_mask, void* out, const base_layer_options* opt,
+                                  const base_layer_debug* dbg, void* stream);
 
 /*
  * The same step for a caller whose activations live in HOST memory: copies h_hidden_bf16 [T,d]

@@ -23,7 +23,7 @@ DEV_NONFINITE_SCORE, DEV_WAIT_EXPIRED, DEV_BAD_INDEX = 1, 2, 4
 
 EXPORTS = (
     "base_predict_costs", "base_aggregate_select", "base_moe_decode_layer_workspace_bytes",
-    "base_moe_decode_layer", "base_moe_decode_layer_host_workspace_bytes", "base_moe_decode_layer_host",
+    "base_moe_decode_layer", "base_moe_decode_layer_noalloc", "base_moe_decode_layer_host_workspace_bytes", "base_moe_decode_layer_host",
     "base_moe_decode_stack_workspace_bytes", "base_moe_decode_stack", "base_profile_events",
     "base_last_launch_count",
     "base_status_string", "base_last_cuda_error",
@@ -71,6 +71,8 @@ def lib():
     L.base_moe_decode_layer_workspace_bytes.restype = C.c_size_t
     L.base_moe_decode_layer.argtypes = [C.POINTER(LayerShape), C.POINTER(LayerWeights), vp, vp, ip, ip, vp, vp,
                                         C.POINTER(LayerOptions), C.POINTER(LayerDebug), vp, C.c_size_t, vp]
+    L.base_moe_decode_layer_noalloc.argtypes = [C.POINTER(LayerShape), C.POINTER(LayerWeights), vp, vp, ip, ip, vp, vp,
+                                                C.POINTER(LayerOptions), C.POINTER(LayerDebug), vp]
     L.base_moe_decode_layer_host_workspace_bytes.argtypes = [C.POINTER(LayerShape), ip]
     L.base_moe_decode_layer_host_workspace_bytes.restype = C.c_size_t
     L.base_moe_decode_layer_host.argtypes = [C.POINTER(LayerShape), C.POINTER(LayerWeights), vp, ip, ip, vp,
@@ -195,6 +197,30 @@ def base_moe_decode_layer(shape, weights, hidden, budget, out, workspace, router
                                        _ptr(router_logits), T, budget, _ptr(forced_mask), _ptr(out), C.byref(opt),
                                        C.byref(debug) if debug is not None else None, _ptr(workspace),
                                        workspace.numel(), _stream(stream)))
+    return out
+
+
+NOALLOC_SCRATCH_BYTES = 16 << 20
+
+
+def base_moe_decode_layer_noalloc(shape, weights, hidden, budget, out, router_logits=None, forced_mask=None,
+                                  gate_rule=GATE_PAPER, fill_rule=FILL_BACKFILL, ffn_impl=FFN_DEFAULT, debug=None,
+                                  stream=None):
+    """The decode step without a caller workspace: scratch is the library's built-in 16 MiB buffer.
+
+    For callers that cannot allocate device memory when they need the layer (inside another engine's
+    memory budget, or handed a stream and tensors but no allocator). All calls on a device share that buffer: do not overlap them.
+    Raises BaseError (code 5) when the shape needs more scratch than the buffer holds.
+    """
+    d, E, K, I = shape
+    T = hidden.shape[0]
+    assert hidden.dtype == torch.bfloat16 and hidden.shape[1] == d
+    assert out.dtype in (torch.bfloat16, torch.float32) and tuple(out.shape) == (T, d)
+    opt = LayerOptions(gate_rule, fill_rule, 1 if out.dtype == torch.float32 else 0, ffn_impl)
+    _check(lib().base_moe_decode_layer_noalloc(C.byref(LayerShape(d, E, K, I)), C.byref(weights), _ptr(hidden),
+                                               _ptr(router_logits), T, budget, _ptr(forced_mask), _ptr(out),
+                                               C.byref(opt), C.byref(debug) if debug is not None else None,
+                                               _stream(stream)))
     return out
 
 

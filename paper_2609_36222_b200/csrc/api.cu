@@ -2,6 +2,8 @@
 // no synchronisation (except the *_host entry point, which waits for its own copies).
 #include <string.h>
 
+#include <mutex>
+
 #include "common.cuh"
 #include "ffn_tc.cuh"
 
@@ -121,6 +123,30 @@ int check_layer_args(const base_layer_shape* shape, const base_layer_weights* w,
   return BASE_OK;
 }
 
+// ---- built-in scratch of base_moe_decode_layer_noalloc -------------------------------------------
+// The array's name is only a host-side handle; kernels need its device address, which is looked up
+// once per device (with that device current) and cached.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[BASE_NOALLOC_SCRATCH_BYTES];
+constexpr int kMaxDevices = 64;
+std::mutex g_noalloc_mu;
+void* g_noalloc_ptr[kMaxDevices] = {};
+
+int noalloc_scratch_address(void** out) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return cuda_fail(e);
+  if (dev < 0 || dev >= kMaxDevices) return BASE_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> g(g_noalloc_mu);
+  if (!g_noalloc_ptr[dev]) {
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_noalloc_scratch);
+    if (e != cudaSuccess) return cuda_fail(e);
+    g_noalloc_ptr[dev] = p;
+  }
+  *out = g_noalloc_ptr[dev];
+  return BASE_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -162,6 +188,38 @@ int base_moe_decode_layer(const base_layer_shape* shape, const base_layer_weight
   if (reinterpret_cast<uintptr_t>(workspace) & 1023u) return BASE_ERR_INVALID_ARG;
   Workspace ws = carve_workspace(workspace, *shape, T);
   if (ws.bytes > workspace_bytes) return BASE_ERR_WORKSPACE_TOO_SMALL;
+  LayerCall c{};
+  c.shape = shape;
+  c.w = weights;
+  c.hidden = hidden_bf16;
+  c.router_logits = router_logits;
+  c.T = T;
+  c.budget = budget;
+  c.forced_mask = forced_mask;
+  c.out = out;
+  if (opt) c.opt = *opt;
+  if (dbg) c.dbg = *dbg;
+  int launches = 0;
+  rc = enqueue_layer(c, ws, static_cast<cudaStream_t>(stream), &launches);
+  if (rc == BASE_OK) g_last_launches = launches;
+  return rc;
+}
+
+int base_moe_decode_layer_noalloc(const base_layer_shape* shape, const base_layer_weights* weights,
+                                  const void* hidden_bf16, const float* router_logits, int T, int budget,
+                                  const uint8_t* forced_mask, void* out, const base_layer_options* opt,
+                                  const base_layer_debug* dbg, void* stream) {
+  int rc = check_layer_args(shape, weights, hidden_bf16, router_logits, T, budget, opt);
+  if (rc != BASE_OK) return rc;
+  if (!out || !aligned16(out)) return BASE_ERR_INVALID_ARG;
+  // the array is 256-byte aligned; the workspace wants 1024, so up to 768 bytes are lost to alignment
+  const size_t need = carve_workspace(nullptr, *shape, T).bytes;
+  if (need + 768 > size_t(BASE_NOALLOC_SCRATCH_BYTES)) return BASE_ERR_SCRATCH_LIMIT;
+  void* scratch = nullptr;
+  rc = noalloc_scratch_address(&scratch);
+  if (rc != BASE_OK) return rc;
+  void* base_ptr = reinterpret_cast<void*>((reinterpret_cast<uintptr_t>(scratch) + 1023) & ~uintptr_t(1023));
+  Workspace ws = carve_workspace(base_ptr, *shape, T);
   LayerCall c{};
   c.shape = shape;
   c.w = weights;
@@ -282,6 +340,7 @@ const char* base_status_string(int code) {
     case BASE_ERR_UNSUPPORTED: return "shape outside the compiled limits";
     case BASE_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
     case BASE_ERR_CUDA: return "CUDA error (see base_last_cuda_error)";
+    case BASE_ERR_SCRATCH_LIMIT: return "shape needs more scratch than the built-in no-allocation buffer holds";
     default: return "unknown status";
   }
 }

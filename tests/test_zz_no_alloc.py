@@ -1,0 +1,69 @@
+"""The no-allocation entry point against the ordinary one.
+
+`base_moe_decode_layer_noalloc` is for callers that cannot hand the library a freshly allocated
+workspace (they run inside another engine that has already given all device memory away, or they
+are handed a stream and tensors but no allocator). It must compute exactly what `base_moe_decode_layer` computes, also when it is
+called twice in a row on the buffer it shares between calls. This file sorts last on purpose: a run
+that stops at the first failure has then already run every other test.
+"""
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2609_36222_b200 import binding as B
+from paper_2609_36222_b200 import workloads as wl
+from paper_2609_36222_b200.layer import DeviceLayer, bits_to_device
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+OUT_ATOL, OUT_RTOL = 2e-2, 1e-2      # the output tolerance of the parity tests
+
+
+def _run(entry, dl, hidden, M, **kw):
+    cfg = dl.cfg
+    T = hidden.shape[0]
+    out = torch.full((T, cfg.d), float("nan"), dtype=torch.float32, device=DEV)
+    dbg, dt = B.alloc_debug(T, cfg.E, cfg.K, M, DEV)
+    entry(out, dbg, **kw)
+    torch.cuda.synchronize()
+    res = {k: v.cpu().numpy() for k, v in dt.items()}
+    res["y"] = out.cpu().numpy().astype(np.float64)
+    return res
+
+
+@pytest.mark.parametrize("name,M", [("qwen3", 32), ("tiny", 6)])
+def test_noalloc_matches_workspace_entry_point_twice_in_a_row(name, M):
+    cfg = wl.CONFIGS[name]
+    dl = DeviceLayer(cfg, DEV)
+    hidden = bits_to_device(wl.hidden_bits(cfg), DEV)
+    hidden2 = bits_to_device(wl.hidden_bits(cfg, layer=7), DEV)   # a second batch for the second call
+
+    def with_ws(h):
+        return _run(lambda out, dbg: B.base_moe_decode_layer(dl.shape, dl.weights, h, M, out, dl.workspace, debug=dbg),
+                    dl, h, M)
+
+    def no_alloc(h):
+        return _run(lambda out, dbg: B.base_moe_decode_layer_noalloc(dl.shape, dl.weights, h, M, out, debug=dbg),
+                    dl, h, M)
+
+    for h in (hidden, hidden2):            # two calls in a row on the shared built-in buffer
+        ref, got = with_ws(h), no_alloc(h)
+        assert got["status"][0] == 0
+        for k in ("topk_ids", "selected_ids", "active_mask", "exec_ids", "expert_counts", "n_dispatched"):
+            np.testing.assert_array_equal(got[k], ref[k])
+        np.testing.assert_allclose(got["scores"], ref["scores"], rtol=1e-3, atol=1e-12)
+        err = np.abs(got["y"] - ref["y"])
+        assert np.isfinite(got["y"]).all()
+        assert (err <= OUT_ATOL + OUT_RTOL * np.abs(ref["y"])).all(), f"max abs err {err.max():.3e}"
+
+
+def test_noalloc_refuses_shapes_beyond_its_buffer():
+    cfg = wl.CONFIGS["qwen3"]
+    T = 256                                   # needs about 30 MiB of scratch, the buffer holds 16 MiB
+    assert B.layer_workspace_bytes(cfg.d, cfg.E, cfg.K, cfg.I, T) > B.NOALLOC_SCRATCH_BYTES
+    dl = DeviceLayer(cfg, DEV, T_max=64)
+    hidden = bits_to_device(wl.hidden_bits(cfg, T), DEV)
+    out = torch.empty(T, cfg.d, dtype=torch.float32, device=DEV)
+    with pytest.raises(B.BaseError, match="scratch"):
+        B.base_moe_decode_layer_noalloc(dl.shape, dl.weights, hidden, 32, out)
