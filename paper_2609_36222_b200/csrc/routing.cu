@@ -152,7 +152,7 @@ cudaError_t launch_aggregate_select(const float* costs, int T, int E, int M, flo
 // applied to both operands and no shared-memory staging is needed. Computing raw for all pairs (not
 // only the routed ones) removes the dependency on the top-K result.
 // ------------------------------------------------------------------------------------------------
-constexpr int kGemvWarps = 4;
+constexpr int kGemvWarps = 8;
 constexpr int kGemvBatch = 8;   // k32-blocks whose loads are in flight together
 
 __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
@@ -222,8 +222,8 @@ __global__ void __launch_bounds__(kGemvWarps * 32) route_scores_kernel(const __n
   s_part[warp][(g + 8) * 8 + 2 * q + 1] = c[3];
   if (q == 0) s_part[warp][128 + g] = zz;
   __syncthreads();
-  {
-    const int i = threadIdx.x;   // 128 threads: one output each
+  if (threadIdx.x < 128) {
+    const int i = threadIdx.x;   // one output each
     float v = 0.f;
 #pragma unroll
     for (int w = 0; w < kGemvWarps; ++w) v += s_part[w][i];
@@ -796,8 +796,54 @@ __global__ void __launch_bounds__(256) combine_kernel(const float* __restrict__ 
   }
 }
 
+// Layer-output-only variant: one thread per four columns, the K row reads of a thread are issued
+// together and nothing is shared between threads, so the kernel is two memory round trips long.
+__global__ void __launch_bounds__(256) combine_out_kernel(const float* __restrict__ ypair,
+                                                          const int32_t* __restrict__ token_slot,
+                                                          const float* __restrict__ gates, void* __restrict__ out,
+                                                          int out_is_fp32, int K, int d) {
+  const int t = blockIdx.x;
+  const int c = (blockIdx.y * 256 + threadIdx.x) * 4;
+  pdl_launch_dependents();
+  pdl_wait();
+  if (c >= d) return;
+  int slot[kMaxK];
+  float g[kMaxK];
+#pragma unroll
+  for (int k = 0; k < kMaxK; ++k) {
+    slot[k] = k < K ? __ldg(token_slot + t * K + k) : -1;
+    g[k] = k < K ? __ldg(gates + t * K + k) : 0.f;
+  }
+  float4 v[kMaxK];
+#pragma unroll
+  for (int k = 0; k < kMaxK; ++k)
+    v[k] = slot[k] >= 0 ? *reinterpret_cast<const float4*>(ypair + size_t(slot[k]) * d + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+  for (int k = 0; k < kMaxK; ++k) {
+    if (slot[k] >= 0) {
+      acc.x = fmaf(g[k], v[k].x, acc.x);
+      acc.y = fmaf(g[k], v[k].y, acc.y);
+      acc.z = fmaf(g[k], v[k].z, acc.z);
+      acc.w = fmaf(g[k], v[k].w, acc.w);
+    }
+  }
+  if (out_is_fp32) {
+    *reinterpret_cast<float4*>(static_cast<float*>(out) + size_t(t) * d + c) = acc;
+  } else {
+    __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
+    uint2 p;
+    p.x = *reinterpret_cast<uint32_t*>(&lo);
+    p.y = *reinterpret_cast<uint32_t*>(&hi);
+    *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(out) + size_t(t) * d + c) = p;
+  }
+}
+
 cudaError_t launch_combine(const Workspace& ws, const void* hidden, void* out, int out_is_fp32, void* x_next,
                            int T, int K, int d, cudaStream_t st) {
+  if (!x_next)
+    return launch_pdl(combine_out_kernel, dim3(T, (d + 1023) / 1024), dim3(256), 0, st, 1, ws.ypair, ws.token_slot,
+                      ws.exec_gates, out, out_is_fp32, K, d);
   return launch_pdl(combine_kernel, dim3(T), dim3(256), 0, st, 1, ws.ypair, ws.token_slot, ws.exec_gates,
                     static_cast<const __nv_bfloat16*>(hidden), out, out_is_fp32, static_cast<__nv_bfloat16*>(x_next), K,
                     d);
