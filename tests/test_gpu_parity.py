@@ -255,3 +255,71 @@ def test_stack_teacher_forced_and_chained():
     # the chained run may take a different discrete route at a near-tie; compare in aggregate
     assert np.median(np.abs(got - x)) < 2e-2
     assert (nd.cpu().numpy() > 0).all() and (nd.cpu().numpy() <= M).all()
+
+
+# ------------------------------------------------------------------------------- bench launch configuration
+
+def test_graph_replay_matches_eager_and_oracle(layers):
+    """The launch configuration bench.py times: the layer captured in a CUDA graph on a side stream and
+    replayed, at the full headline size; outputs bit-identical to the eager call and within tolerance of the oracle."""
+    host, dl = layers("qwen3")
+    cfg = host.cfg
+    hid = bits_to_device(host.hidden_bits, DEV)
+    eager = torch.empty(cfg.T, cfg.d, dtype=torch.bfloat16, device=DEV)
+    B.base_moe_decode_layer(dl.shape, dl.weights, hid, 32, eager, dl.workspace)
+    torch.cuda.synchronize()
+    out = torch.zeros_like(eager)
+    stream = torch.cuda.Stream()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        B.base_moe_decode_layer(dl.shape, dl.weights, hid, 32, out, dl.workspace, stream=stream)   # warm-up
+    stream.synchronize()
+    with torch.cuda.graph(g, stream=stream):
+        B.base_moe_decode_layer(dl.shape, dl.weights, hid, 32, out, dl.workspace, stream=stream)
+    for _ in range(3):
+        out.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(out, eager)
+    logits = O.router_logits(host.z, host.router_w, host.router_bias)
+    ref = O.moe_decode_layer(host.z, logits, host.pred_A, host.pred_b, host.expert_weights, cfg.K, 32)
+    # the device routes on its own logits here; compare outputs only where the routes agree
+    got = run_gpu(dl, hid, 32)
+    same = (got["exec_ids"] == ref["exec_ids"]).all(axis=1)
+    assert same.mean() > 0.9
+    y = out.float().cpu().numpy().astype(np.float64)
+    err = np.abs(y - ref["y"])[same]
+    assert (err <= 2e-2 + 1e-2 * np.abs(ref["y"][same])).all()
+
+
+def test_fitted_predictor_mid_config():
+    """The mid config with its predictor least-squares fitted on seeded calibration tokens against the oracle's
+    brute-force removal costs; the fitted coefficients (rounded to bf16 / fp32) are given to both paths."""
+    cfg = wl.CONFIGS["mid"]
+    host = HostLayer(cfg)
+    n_cal = 4096                                       # seeded synthetic calibration tokens
+    zc = wl.bf16_bits_to_f64(wl.hidden_bits(cfg, n_cal, stream="calib"))
+    lc = O.router_logits(zc, host.router_w, host.router_bias)
+    A, b = O.fit_predictor(zc, lc, host.expert_weights, cfg.K, cfg.E, lam=1e-2)
+    A_bits = wl.f32_to_bf16_bits(A.astype(np.float32)).reshape(cfg.E, cfg.d)
+    host.small["pred_A"] = A_bits
+    host.small["pred_b"] = b.astype(np.float32)
+    dl = device_layer_from_host(host, DEV)
+    assert np.abs(b).max() < 20 and np.isfinite(A).all()
+    for M in (8, 24):
+        rep = check_layer(host, dl, M)
+        # the fitted intercepts are far from zero (log-energies), so the scores differ from the sum of w^2
+        assert np.abs(np.log(rep["ref"]["scores"][rep["ref"]["scores"] > 0])).max() > 1.0
+
+
+@pytest.mark.parametrize("T,M", [(1, 16), (8, 32), (32, 64), (128, 32), (256, 16), (256, 64)])
+def test_stack_shape_batch_and_budget_sweep(T, M):
+    """One full-size layer of the 48-layer stack workload at the batch sizes and budgets of its sweep
+    (batch 1 ... 256 selects the 32-, 64- and 128-token tile variants of the FFN kernel)."""
+    cfg = wl.CONFIGS["qwen3_stack"]
+    host = HostLayer(cfg, layer=5 + T % 7, T=T)
+    dl = device_layer_from_host(host, DEV)
+    rep = check_layer(host, dl, M)
+    assert rep["n_dispatched"] <= min(M, cfg.E)
+    del dl
+    torch.cuda.empty_cache()
