@@ -278,23 +278,36 @@ def run_ours(args, cfg, T, M):
     ms = multi.max_over_ranks(ms, dist, dev)
 
     # ---- per-kernel pass for the roofline: the library records the caller's events around the FFN kernels
-    n_prof = min(args.steps, 40)
+    # Six events per replica are recorded by the library between the kernels of the step; the step is captured
+    # in a graph with those records as nodes, so the replay has no host launch gaps.
+    n_prof = min(args.steps, 60)
     ffn_us, stage_us = None, None
     if not args.profile:
-        evs = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(n_prof)]
-        with torch.cuda.stream(stream):
-            for i in range(3):
-                step_eager(i)
-            for i, ev in enumerate(evs):
-                for e in ev:
+        n_g = 1 if stack else n_rep
+        evs = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(n_g)]
+        pgraphs = []
+        for r in range(n_g):
+            with torch.cuda.stream(stream):
+                for e in evs[r]:
                     e.record(stream)          # create the handles before the library records them again
-                B.set_profile_events(ev)
-                step_eager(3 + i)
-            B.set_profile_events(None)
-        stream.synchronize()
+            stream.synchronize()
+            B.set_profile_events(evs[r])
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                step_eager(r)
+            pgraphs.append(g)
+        B.set_profile_events(None)
+        samples = {name: [] for name in B.PROFILE_STAGES}
+        with torch.cuda.stream(stream):
+            for i in range(3 + n_prof):
+                r = i % n_g
+                pgraphs[r].replay()
+                stream.synchronize()
+                if i >= 3:
+                    for j, name in enumerate(B.PROFILE_STAGES):
+                        samples[name].append(evs[r][j].elapsed_time(evs[r][j + 1]) * 1e3)
         # (in a stack every layer re-records the events, so these are the last layer's kernels)
-        stage_us = {name: statistics.mean(ev[j].elapsed_time(ev[j + 1]) for ev in evs) * 1e3
-                    for j, name in enumerate(B.PROFILE_STAGES)}
+        stage_us = {name: statistics.mean(v) for name, v in samples.items()}
         ffn_us = stage_us["expert_ffn"]
 
     # ---- unlimited budget (dense batch-union step) for the speed-up, same protocol

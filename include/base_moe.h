@@ -217,7 +217,8 @@ int base_moe_decode_stack(const base_layer_shape* shape, const base_layer_weight
  * stream: [0] before the first kernel, [1] after the router/predictor GEMV, [2] after the routing
  * kernel, [3] after the gather, [4] after the expert-FFN kernels, [5] after the combine. A benchmark
  * can thus time each kernel inside a full step. The array is copied; pass NULL to switch the hook
- * off. Not for use during stream capture.
+ * off. When the stream is being captured the records become graph nodes (recorded with the external
+ * flag), so a replay of the graph times the kernels without host launch gaps.
  */
 #define BASE_PROFILE_EVENTS 6
 int base_profile_events(void* const* events);

@@ -17,7 +17,13 @@ thread_local cudaEvent_t g_ev[BASE_PROFILE_EVENTS] = {};
 thread_local bool g_ev_on = false;
 
 inline void mark(int i, cudaStream_t st) {
-  if (g_ev_on && g_ev[i]) cudaEventRecord(g_ev[i], st);
+  if (!g_ev_on || !g_ev[i]) return;
+  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+  cudaStreamIsCapturing(st, &cap);
+  // inside a capture the record becomes a graph node; the external flag keeps the event usable
+  // for cudaEventElapsedTime after a replay
+  if (cap == cudaStreamCaptureStatusActive) cudaEventRecordWithFlags(g_ev[i], st, cudaEventRecordExternal);
+  else cudaEventRecord(g_ev[i], st);
 }
 
 inline int cuda_fail(cudaError_t e) {
