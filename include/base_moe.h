@@ -53,6 +53,11 @@ enum {                             /* bits of the device status word */
 
 enum { BASE_GATE_PAPER = 0,        /* Sec. 3.5: original top-K denominator (gates may sum to < 1) */
        BASE_GATE_RENORM = 1 };     /* renormalise over the executed experts (OEA-style variant) */
+enum { BASE_SCORE_PREDICTED = 0,   /* Eq. log_energy_predictor: sum of w^2 exp(a.z/|z| + b) (the method) */
+       BASE_SCORE_WEIGHT_SQ = 1,   /* squared router-weight sum, sum of w^2   (App. Selection-Rule Ablation) */
+       BASE_SCORE_WEIGHT = 2,      /* router-weight sum, sum of w */
+       BASE_SCORE_STATIC = 3,      /* static energy, sum of w^2 mu_u with mu_u = exp(pred_b[u]) */
+       BASE_SCORE_TOP1_UNION = 4 };/* number of tokens whose first choice the expert is (positive on the top-1 union) */
 enum { BASE_FILL_BACKFILL = 0,     /* Sec. 3.5: next-preferred experts inside the active set */
        BASE_FILL_DROP = 1 };       /* fill-rule ablation: unavailable routes are removed */
 
@@ -122,6 +127,7 @@ typedef struct {
   int fill_rule;            /* BASE_FILL_* */
   int out_is_fp32;          /* 0: out is bf16 [T,d]; 1: out is fp32 [T,d] */
   int ffn_impl;             /* 0: default (tensor-core streaming kernels); 1: simple CUDA-core kernels */
+  int score_rule;           /* BASE_SCORE_*: what a routed pair contributes to its expert's batch score */
 } base_layer_options;
 
 /* Bytes of device workspace base_moe_decode_layer needs for up to T_max tokens (0 on bad shape). */

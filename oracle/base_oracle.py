@@ -27,6 +27,12 @@ GATE_RULE_PAPER = 0       # Sec. 3.5: denominator from the token's ORIGINAL top-
 GATE_RULE_RENORM = 1      # OEA-style: renormalise over the executed experts
 FILL_BACKFILL = 0         # Sec. 3.5: next-preferred experts inside the active set
 FILL_DROP = 1             # fill-rule ablation: unavailable routes are simply removed
+# what a routed pair contributes to its expert's batch score (App. Selection-Rule Ablation)
+SCORE_PREDICTED = 0       # w^2 exp(a . z-bar + b): the method (Eq. log_energy_predictor)
+SCORE_WEIGHT_SQ = 1       # squared router-weight sum
+SCORE_WEIGHT = 2          # router-weight sum
+SCORE_STATIC = 3          # static energy w^2 mu_u, with mu_u = exp(b_u)
+SCORE_TOP1_UNION = 4      # 1 per token whose first choice the expert is (positive exactly on the top-1 union)
 
 
 # ----------------------------------------------------------------------------- router (Sec. 3.1)
@@ -69,8 +75,10 @@ def normalise(z):
     return z / np.maximum(n, 1e-30)
 
 
-def predict_costs(z, R, w, pred_A, pred_b):
-    """c[t,u] = w_{t,u}^2 * exp(a_u . z-bar_t + b_u) for u in R_t, 0 elsewhere. Shape [T,E]."""
+def predict_costs(z, R, w, pred_A, pred_b, score_rule=SCORE_PREDICTED):
+    """c[t,u] = w_{t,u}^2 * exp(a_u . z-bar_t + b_u) for u in R_t, 0 elsewhere. Shape [T,E].
+
+    ``score_rule`` swaps the contribution for one of the ablation scores of App. Selection-Rule Ablation."""
     zbar = normalise(z)
     A = np.asarray(pred_A, np.float64)
     b = np.asarray(pred_b, np.float64)
@@ -81,8 +89,19 @@ def predict_costs(z, R, w, pred_A, pred_b):
             u = int(R[t, k])
             if u < 0:
                 continue
-            s_hat = float(A[u] @ zbar[t]) + b[u]
-            costs[t, u] = w[t, k] ** 2 * np.exp(s_hat)
+            if score_rule == SCORE_PREDICTED:
+                s_hat = float(A[u] @ zbar[t]) + b[u]
+                costs[t, u] = w[t, k] ** 2 * np.exp(s_hat)
+            elif score_rule == SCORE_WEIGHT_SQ:
+                costs[t, u] = w[t, k] ** 2
+            elif score_rule == SCORE_WEIGHT:
+                costs[t, u] = w[t, k]
+            elif score_rule == SCORE_STATIC:
+                costs[t, u] = w[t, k] ** 2 * np.exp(b[u])
+            elif score_rule == SCORE_TOP1_UNION:
+                costs[t, u] = 1.0 if k == 0 else 0.0
+            else:
+                raise ValueError(score_rule)
     return costs
 
 
@@ -156,7 +175,7 @@ def execute(z, ids, gates, expert_weights):
 # ----------------------------------------------------------------------------- the layer
 
 def moe_decode_layer(z, logits, pred_A, pred_b, expert_weights, K, M,
-                     gate_rule=GATE_RULE_PAPER, fill=FILL_BACKFILL, forced_mask=None):
+                     gate_rule=GATE_RULE_PAPER, fill=FILL_BACKFILL, forced_mask=None, score_rule=SCORE_PREDICTED):
     """One BASE decode step of one MoE layer, in the paper's order:
     route -> predict costs -> aggregate -> top-M -> restrict routes -> execute.
 
@@ -164,7 +183,7 @@ def moe_decode_layer(z, logits, pred_A, pred_b, expert_weights, K, M,
     Returns a dict with every intermediate.
     """
     order, R, q, S, w = route_topk(logits, K)
-    costs = predict_costs(z, R, w, pred_A, pred_b)
+    costs = predict_costs(z, R, w, pred_A, pred_b, score_rule)
     scores = aggregate(costs)
     sel, mask = select_top(scores, M)
     if forced_mask is not None:

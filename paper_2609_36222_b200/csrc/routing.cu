@@ -374,13 +374,16 @@ __global__ void __launch_bounds__(kRoutingThreads) routing_kernel(RoutingArgs a)
     }
     const uint32_t avail0 = avail;
     float m = 0.f, myv = 0.f;
-    int myid = kNone;
+    int myid = kNone, first_id = kNone;
     for (int k = 0; k < K; ++k) {
       uint32_t gk;
       int gi;
       take_best<NV>(key, avail, lane, gk, gi);
       const float bv = key_float(gk);
-      if (k == 0) m = (gi != kNone && bv > -INFINITY) ? bv : 0.f;
+      if (k == 0) {
+        m = (gi != kNone && bv > -INFINITY) ? bv : 0.f;
+        first_id = gi;
+      }
       if (lane == k) {
         myv = bv;
         myid = gi;
@@ -401,7 +404,13 @@ __global__ void __launch_bounds__(kRoutingThreads) routing_kernel(RoutingArgs a)
         float c = 0.f;
         if ((taken >> i) & 1u) {
           const float w = S_t > 0.f ? q[i] / S_t : 0.f;
-          c = w * w * expf(sh[i]);
+          switch (a.score_rule) {
+            case BASE_SCORE_WEIGHT_SQ: c = w * w; break;
+            case BASE_SCORE_WEIGHT: c = w; break;
+            case BASE_SCORE_STATIC: c = w * w * expf(a.pred_b[e]); break;
+            case BASE_SCORE_TOP1_UNION: c = (e == first_id) ? 1.f : 0.f; break;
+            default: c = w * w * expf(sh[i]); break;
+          }
         }
         a.ws.costs[size_t(t) * E + e] = c;
       }

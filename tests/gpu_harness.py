@@ -49,15 +49,16 @@ def run_gpu(dl, hidden_dev, M, logits=None, forced_mask=None, out_dtype=torch.fl
     return res
 
 
-def check_layer(host, dl, M, gate_rule=0, fill_rule=0, out_dtype=torch.float32, ffn_impl=0, check_out=True):
+def check_layer(host, dl, M, gate_rule=0, fill_rule=0, out_dtype=torch.float32, ffn_impl=0, check_out=True,
+                score_rule=0):
     """Run oracle and CUDA path on the same inputs and compare every intermediate. Returns a report."""
     cfg = host.cfg
     z = host.z
     logits = O.router_logits(z, host.router_w, host.router_bias)
     ref = O.moe_decode_layer(z, logits, host.pred_A, host.pred_b, host.expert_weights, cfg.K, M,
-                             gate_rule=gate_rule, fill=fill_rule)
+                             gate_rule=gate_rule, fill=fill_rule, score_rule=score_rule)
     hidden_dev = bits_to_device(host.hidden_bits, dl.device)
-    kw = dict(gate_rule=gate_rule, fill_rule=fill_rule, ffn_impl=ffn_impl, out_dtype=out_dtype)
+    kw = dict(gate_rule=gate_rule, fill_rule=fill_rule, ffn_impl=ffn_impl, out_dtype=out_dtype, score_rule=score_rule)
     got = run_gpu(dl, hidden_dev, M, logits=logits, **kw)
 
     assert got["status"][0] == 0

@@ -323,3 +323,13 @@ def test_stack_shape_batch_and_budget_sweep(T, M):
     assert rep["n_dispatched"] <= min(M, cfg.E)
     del dl
     torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("rule", [B.SCORE_WEIGHT_SQ, B.SCORE_WEIGHT, B.SCORE_STATIC, B.SCORE_TOP1_UNION])
+def test_selection_score_variants(layers, rule):
+    """The ablation scores of App. Selection-Rule Ablation behind `score_rule`, same parity bar."""
+    host, dl = layers("qwen3")
+    rep = check_layer(host, dl, 32, score_rule=rule)
+    if rule == B.SCORE_TOP1_UNION:
+        top1 = set(rep["ref"]["R"][:, 0].tolist())
+        assert set(np.nonzero(rep["ref"]["scores"])[0].tolist()) == top1

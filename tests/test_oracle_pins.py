@@ -361,3 +361,30 @@ def test_fit_predictor_against_brute_force_removal_costs():
     pc = np.take_along_axis(O.predict_costs(z[:1000], Rc, wc, A, b), Rc, axis=1) / wc ** 2
     for u in range(E):
         assert pc[Rc == u].mean() == pytest.approx(tc[Rc == u].mean(), rel=1e-9)
+
+
+def test_ablation_scores_closed_forms():
+    """The router-only and static scores of App. Selection-Rule Ablation, checked against direct sums; the
+    squared-weight and static scores are also the predictor with a = 0 (b = 0, resp. b = log mu)."""
+    z, logits, A, b, ew = make_layer(21, T=9)
+    K, E = 3, logits.shape[1]
+    _, R, _, _, w = O.route_topk(logits, K)
+    def direct(f):
+        s = np.zeros(E)
+        for t in range(R.shape[0]):
+            for k in range(K):
+                s[R[t, k]] += f(t, k)
+        return s
+    sq = O.aggregate(O.predict_costs(z, R, w, A, b, O.SCORE_WEIGHT_SQ))
+    np.testing.assert_allclose(sq, direct(lambda t, k: w[t, k] ** 2), rtol=1e-14)
+    np.testing.assert_allclose(sq, O.aggregate(O.predict_costs(z, R, w, 0 * A, 0 * b)), rtol=1e-14)
+    np.testing.assert_allclose(O.aggregate(O.predict_costs(z, R, w, A, b, O.SCORE_WEIGHT)),
+                               direct(lambda t, k: w[t, k]), rtol=1e-14)
+    st = O.aggregate(O.predict_costs(z, R, w, A, b, O.SCORE_STATIC))
+    np.testing.assert_allclose(st, direct(lambda t, k: w[t, k] ** 2 * np.exp(b[R[t, k]])), rtol=1e-13)
+    np.testing.assert_allclose(st, O.aggregate(O.predict_costs(z, R, w, 0 * A, b)), rtol=1e-13)
+    u1 = O.aggregate(O.predict_costs(z, R, w, A, b, O.SCORE_TOP1_UNION))
+    assert set(np.nonzero(u1)[0].tolist()) == set(R[:, 0].tolist())
+    assert u1.sum() == R.shape[0]
+    # weights of one token sum to one, so the router-weight scores sum to the batch size
+    assert O.aggregate(O.predict_costs(z, R, w, A, b, O.SCORE_WEIGHT)).sum() == pytest.approx(R.shape[0], rel=1e-12)
