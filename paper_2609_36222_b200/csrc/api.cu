@@ -99,7 +99,7 @@ int enqueue_layer(const LayerCall& c, const Workspace& ws, cudaStream_t st, int*
   if (c.opt.ffn_impl == 1) {
     e = launch_ffn_simple(s, *c.w, ws, st, launches);
   } else {
-    e = launch_ffn_tc(s, *c.w, c.hidden, ws, c.T, st, launches);
+    e = launch_ffn_tc(s, *c.w, c.hidden, ws, c.T, c.budget, st, launches);
   }
   if (e != cudaSuccess) return cuda_fail(e);
   mark(4, st);

@@ -29,6 +29,7 @@
 // is freed and BASE_DEV_WAIT_EXPIRED is OR-ed into the status word.
 #include <cuda.h>
 
+#include <algorithm>
 #include <mutex>
 #include <unordered_map>
 
@@ -72,6 +73,7 @@ struct Plan {
 // always on work that never waits itself.
 struct Unit {
   int phase, seg, expert, offset, count, npad, tile;
+  int kb0;   // first k-block of the unit's K range (down units of a split tile start later)
 };
 
 struct Bars {
@@ -106,7 +108,9 @@ struct FfnParams {
   const int32_t* slot_token;     // [rows] token of every sorted row
   int I, d;
   int tiles1, tiles2;   // work units per segment: I/64 gate/up tiles, d/128 down tiles
-  int steps1, steps2;   // pipeline stages per unit: ceil(d/64 / 2), ceil(I/64 / 2)
+  int steps1, steps2;   // pipeline stages per unit: ceil(d/64 / 2), ceil(kb2 / 2)
+  int ksplit;           // down pass: each tile's K range (I) is split over this many units (1 or 2)
+  int kb2;              // down pass: k-blocks per unit = ceil(I/64 / ksplit), even
   int split_a;          // gate/up pass: 1 = gate and up come from two maps (two boxes per k-block)
 };
 
@@ -237,10 +241,15 @@ __device__ __forceinline__ Unit decode_unit(const FfnParams& p, int u, int n_seg
   const int u1 = n_seg * p.tiles1;
   r.phase = u < u1 ? 1 : 2;
   const int v = u < u1 ? u : u - u1;
-  const int tiles = u < u1 ? p.tiles1 : p.tiles2;
+  const int tiles = u < u1 ? p.tiles1 : p.tiles2 * p.ksplit;
   const int seg = v / tiles;
   r.seg = seg;
   r.tile = v - seg * tiles;
+  r.kb0 = 0;
+  if (u >= u1 && p.ksplit > 1) {   // (tile, half) pairs: neighbouring units share the token rows in L2
+    r.kb0 = (r.tile % p.ksplit) * p.kb2;
+    r.tile /= p.ksplit;
+  }
   r.expert = p.seg_expert[seg];
   r.offset = p.seg_offset[seg];
   r.count = p.seg_count[seg];
@@ -295,7 +304,7 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
   // Everything above is independent of the routing result and overlaps the previous kernels.
   pdl_wait();
   const int n_seg = p.counters[kCtrSegments];
-  const int n_units = n_seg * (p.tiles1 + p.tiles2);
+  const int n_units = n_seg * (p.tiles1 + p.tiles2 * p.ksplit);
   const int n_slots = p.counters[kCtrSlots];
   tcgen05_fence_before();
   __syncthreads();
@@ -326,13 +335,13 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
         // or the h rows of the segment (down units). Weight boxes do not depend on it and go first.
         bool b_ready = gu ? x_ready : false;
         const int32_t* flag = gu ? p.counters + kCtrGather : p.counters + kCtrReady + un.seg;
-        const int need = gu ? n_slots : p.tiles1;
+        const int need = gu ? n_slots + (p.ksplit > 1 ? int(gridDim.x) : 0) : p.tiles1;
         for (int st = 0; st < n_steps; ++st) {
           if (!mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1u, abort_flag)) {
             ok = false;
             break;
           }
-          const int kb = st * kKbPerStage;
+          const int kb = un.kb0 + st * kKbPerStage;
           const uint32_t full = smem_u32(&bars->full[stage]);
           const uint32_t sa = smem_u32(stages + size_t(stage) * kStageBytes);
           const uint32_t sb = sa + kStageABytes;
@@ -406,7 +415,7 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
           break;
         }
         const int n_steps = un.phase == 1 ? p.steps1 : p.steps2;
-        const int kblocks = un.phase == 1 ? kblocks1 : kblocks2;
+        const int kblocks = un.phase == 1 ? kblocks1 : min(kblocks2 - un.kb0, p.kb2);
         const uint32_t d_tmem = tmem_base + uint32_t(acc * kAccCols);
         const uint32_t idesc = make_idesc(un.npad);
         const uint32_t tile_b = uint32_t(un.npad * 128);
@@ -474,6 +483,17 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
         if (lane == 0) red_release_add(p.counters + kCtrGather, 1);
       }
     }
+    if (p.ksplit > 1) {
+      // the two halves of a split down tile add into ypair, which therefore starts from zero; every
+      // CTA clears its share and reports it through the same counter as the gather
+      const size_t n4 = size_t(n_slots) * p.d / 4;
+      float4* y4 = reinterpret_cast<float4*>(p.ypair);
+      for (size_t i = size_t(blockIdx.x) * 128 + (threadIdx.x - 64); i < n4; i += size_t(gridDim.x) * 128)
+        y4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+      __threadfence();
+      named_sync(5, 128);
+      if (threadIdx.x == 64) red_release_add(p.counters + kCtrGather, 1);
+    }
     int acc = 0;
     uint32_t acc_phase = 0;
     while (true) {
@@ -528,8 +548,13 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
           float v[16];
           tmem_ld16(taddr + c0, v);
 #pragma unroll
-          for (int c = 0; c < 16; ++c)
-            if (c0 + c < un.count) yrow[size_t(c0 + c) * p.d] = v[c];
+          for (int c = 0; c < 16; ++c) {
+            if (c0 + c < un.count) {
+              // a split tile has two contributions per element; 0 + a + b does not depend on their order
+              if (p.ksplit > 1) atomicAdd(yrow + size_t(c0 + c) * p.d, v[c]);
+              else yrow[size_t(c0 + c) * p.d] = v[c];
+            }
+          }
         }
         tcgen05_fence_before();
         mbar_arrive(smem_u32(&bars->acc_empty[acc]));
@@ -694,7 +719,7 @@ cudaError_t launch_kernel(const MapSet& m1, const MapSet& m2, const FfnParams& p
 }  // namespace
 
 cudaError_t launch_ffn_tc(const base_layer_shape& s, const base_layer_weights& w, const void* hidden,
-                          const Workspace& ws, int T, cudaStream_t st, int* launches) {
+                          const Workspace& ws, int T, int budget, cudaStream_t st, int* launches) {
   const uint64_t slots = uint64_t(T) * s.K + kRowPad;
   const uint64_t wrows = uint64_t(s.E) * s.I;
   MapSet m1{}, m2{};
@@ -730,8 +755,13 @@ cudaError_t launch_ffn_tc(const base_layer_shape& s, const base_layer_weights& w
   p.tiles1 = s.I / 64;
   p.tiles2 = s.d / 128;
   p.steps1 = (s.d / kBlockK + int(kKbPerStage) - 1) / int(kKbPerStage);
-  p.steps2 = (s.I / kBlockK + int(kKbPerStage) - 1) / int(kKbPerStage);
-  const int max_units = segs * (p.tiles1 + p.tiles2);
+  // Few experts with long down rows (d/128 tiles each) leave SMs without a down unit; split K in two then.
+  const int kb_all = s.I / kBlockK;
+  const int expect_experts = std::min(std::min(budget, s.E), T * s.K);
+  p.ksplit = (p.tiles2 * expect_experts < sm_count() && kb_all >= 8) ? 2 : 1;
+  p.kb2 = p.ksplit == 1 ? kb_all : ((kb_all + 1) / 2 + int(kKbPerStage) - 1) / int(kKbPerStage) * int(kKbPerStage);
+  p.steps2 = (p.kb2 + int(kKbPerStage) - 1) / int(kKbPerStage);
+  const int max_units = segs * (p.tiles1 + p.tiles2 * p.ksplit);
   // No expert can receive more tokens than the batch holds, which bounds the token tile.
   cudaError_t e;
   if (T <= 32) e = launch_kernel<32>(m1, m2, p, max_units, st);

@@ -333,3 +333,13 @@ def test_selection_score_variants(layers, rule):
     if rule == B.SCORE_TOP1_UNION:
         top1 = set(rep["ref"]["R"][:, 0].tolist())
         assert set(np.nonzero(rep["ref"]["scores"])[0].tolist()) == top1
+
+
+def test_split_down_pass_is_deterministic(layers):
+    """Few dispatched experts (mid config, budget 8) make the down pass split its K range in two halves that
+    add into the same output element; the result must not depend on which half arrives first."""
+    host, dl = layers("mid")
+    hid = bits_to_device(host.hidden_bits, DEV)
+    runs = [run_gpu(dl, hid, 8)["y"] for _ in range(4)]
+    for y in runs[1:]:
+        np.testing.assert_array_equal(y, runs[0])
