@@ -13,7 +13,8 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libbase_moe.so")
+# BASE_MOE_LIB selects another build of the library (A/B measurements); the default is the in-tree build.
+LIB_PATH = os.environ.get("BASE_MOE_LIB") or os.path.join(_HERE, "libbase_moe.so")
 
 BASE_OK = 0
 GATE_PAPER, GATE_RENORM = 0, 1

@@ -236,19 +236,20 @@ __device__ __forceinline__ bool named_and(int id, int threads, bool pred) {
   return out != 0;
 }
 
+template <int kSplit>
 __device__ __forceinline__ Unit decode_unit(const FfnParams& p, int u, int n_seg) {
   Unit r;
   const int u1 = n_seg * p.tiles1;
   r.phase = u < u1 ? 1 : 2;
   const int v = u < u1 ? u : u - u1;
-  const int tiles = u < u1 ? p.tiles1 : p.tiles2 * p.ksplit;
+  const int tiles = u < u1 ? p.tiles1 : p.tiles2 * kSplit;
   const int seg = v / tiles;
   r.seg = seg;
   r.tile = v - seg * tiles;
   r.kb0 = 0;
-  if (u >= u1 && p.ksplit > 1) {   // (tile, half) pairs: neighbouring units share the token rows in L2
-    r.kb0 = (r.tile % p.ksplit) * p.kb2;
-    r.tile /= p.ksplit;
+  if (kSplit > 1 && u >= u1) {   // (tile, half) pairs: neighbouring units share the token rows in L2
+    r.kb0 = (r.tile % kSplit) * p.kb2;
+    r.tile /= kSplit;
   }
   r.expert = p.seg_expert[seg];
   r.offset = p.seg_offset[seg];
@@ -267,7 +268,7 @@ __device__ __forceinline__ void red_release_add(int32_t* ptr, int v) {
   asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(ptr), "r"(v) : "memory");
 }
 
-template <int kMaxN>
+template <int kMaxN, int kSplit>
 __global__ void __launch_bounds__(kThreads, 1)
 ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapSet maps2, const FfnParams p) {
   using P = Plan<kMaxN>;
@@ -304,7 +305,7 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
   // Everything above is independent of the routing result and overlaps the previous kernels.
   pdl_wait();
   const int n_seg = p.counters[kCtrSegments];
-  const int n_units = n_seg * (p.tiles1 + p.tiles2 * p.ksplit);
+  const int n_units = n_seg * (p.tiles1 + p.tiles2 * kSplit);
   const int n_slots = p.counters[kCtrSlots];
   tcgen05_fence_before();
   __syncthreads();
@@ -322,7 +323,7 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
       // the ticket and the decoding of the next unit are requested one unit ahead, so their memory
       // latency never stalls the weight stream
       int u_cur = atomicAdd(p.counters + kCtrTicket, 1);
-      Unit un_next = decode_unit(p, min(u_cur, max(n_units - 1, 0)), n_seg);
+      Unit un_next = decode_unit<kSplit>(p, min(u_cur, max(n_units - 1, 0)), n_seg);
       while (ok && u_cur < n_units) {
         const Unit un = un_next;
         int u_next = n_units;
@@ -335,13 +336,13 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
         // or the h rows of the segment (down units). Weight boxes do not depend on it and go first.
         bool b_ready = gu ? x_ready : false;
         const int32_t* flag = gu ? p.counters + kCtrGather : p.counters + kCtrReady + un.seg;
-        const int need = gu ? n_slots + (p.ksplit > 1 ? int(gridDim.x) : 0) : p.tiles1;
+        const int need = gu ? n_slots + (kSplit > 1 ? int(gridDim.x) : 0) : p.tiles1;
         for (int st = 0; st < n_steps; ++st) {
           if (!mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1u, abort_flag)) {
             ok = false;
             break;
           }
-          const int kb = un.kb0 + st * kKbPerStage;
+          const int kb = (kSplit > 1 ? un.kb0 : 0) + st * kKbPerStage;
           const uint32_t full = smem_u32(&bars->full[stage]);
           const uint32_t sa = smem_u32(stages + size_t(stage) * kStageBytes);
           const uint32_t sb = sa + kStageABytes;
@@ -387,7 +388,7 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
             stage = 0;
             phase ^= 1u;
           }
-          if (st == 0 && u_next < n_units) un_next = decode_unit(p, u_next, n_seg);
+          if (st == 0 && u_next < n_units) un_next = decode_unit<kSplit>(p, u_next, n_seg);
         }
         u_cur = u_next;
       }
@@ -415,7 +416,7 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
           break;
         }
         const int n_steps = un.phase == 1 ? p.steps1 : p.steps2;
-        const int kblocks = un.phase == 1 ? kblocks1 : min(kblocks2 - un.kb0, p.kb2);
+        const int kblocks = un.phase == 1 ? kblocks1 : (kSplit > 1 ? min(kblocks2 - un.kb0, p.kb2) : kblocks2);
         const uint32_t d_tmem = tmem_base + uint32_t(acc * kAccCols);
         const uint32_t idesc = make_idesc(un.npad);
         const uint32_t tile_b = uint32_t(un.npad * 128);
@@ -483,7 +484,7 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
         if (lane == 0) red_release_add(p.counters + kCtrGather, 1);
       }
     }
-    if (p.ksplit > 1) {
+    if (kSplit > 1) {
       // the two halves of a split down tile add into ypair, which therefore starts from zero; every
       // CTA clears its share and reports it through the same counter as the gather
       const size_t n4 = size_t(n_slots) * p.d / 4;
@@ -544,16 +545,22 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
         }
       } else {
         float* yrow = p.ypair + size_t(un.offset) * p.d + un.tile * 128 + q * 32 + lane;
-        for (int c0 = 0; c0 < un.npad; c0 += 16) {
-          float v[16];
-          tmem_ld16(taddr + c0, v);
+        if (kSplit == 1) {
+          for (int c0 = 0; c0 < un.npad; c0 += 16) {
+            float v[16];
+            tmem_ld16(taddr + c0, v);
 #pragma unroll
-          for (int c = 0; c < 16; ++c) {
-            if (c0 + c < un.count) {
-              // a split tile has two contributions per element; 0 + a + b does not depend on their order
-              if (p.ksplit > 1) atomicAdd(yrow + size_t(c0 + c) * p.d, v[c]);
-              else yrow[size_t(c0 + c) * p.d] = v[c];
-            }
+            for (int c = 0; c < 16; ++c)
+              if (c0 + c < un.count) yrow[size_t(c0 + c) * p.d] = v[c];
+          }
+        } else {
+          // a split tile has two contributions per element; 0 + a + b does not depend on their order
+          for (int c0 = 0; c0 < un.npad; c0 += 16) {
+            float v[16];
+            tmem_ld16(taddr + c0, v);
+#pragma unroll
+            for (int c = 0; c < 16; ++c)
+              if (c0 + c < un.count) atomicAdd(yrow + size_t(c0 + c) * p.d, v[c]);
           }
         }
         tcgen05_fence_before();
@@ -707,13 +714,21 @@ int sm_count() {
   return n;
 }
 
-template <int kMaxN>
-cudaError_t launch_kernel(const MapSet& m1, const MapSet& m2, const FfnParams& p, int max_units, cudaStream_t st) {
-  static cudaError_t attr = cudaFuncSetAttribute(ffn_tc_kernel<kMaxN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+template <int kMaxN, int kSplit>
+cudaError_t launch_variant(const MapSet& m1, const MapSet& m2, const FfnParams& p, int max_units, cudaStream_t st) {
+  static cudaError_t attr = cudaFuncSetAttribute(ffn_tc_kernel<kMaxN, kSplit>,
+                                                 cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                  int(Plan<kMaxN>::kSmemBytes));
   if (attr != cudaSuccess) return attr;
   const int grid = min(sm_count(), max_units);
-  return launch_pdl(ffn_tc_kernel<kMaxN>, dim3(grid), dim3(kThreads), Plan<kMaxN>::kSmemBytes, st, 1, m1, m2, p);
+  return launch_pdl(ffn_tc_kernel<kMaxN, kSplit>, dim3(grid), dim3(kThreads), Plan<kMaxN>::kSmemBytes, st, 1, m1, m2,
+                    p);
+}
+
+template <int kMaxN>
+cudaError_t launch_kernel(const MapSet& m1, const MapSet& m2, const FfnParams& p, int max_units, cudaStream_t st) {
+  return p.ksplit > 1 ? launch_variant<kMaxN, 2>(m1, m2, p, max_units, st)
+                      : launch_variant<kMaxN, 1>(m1, m2, p, max_units, st);
 }
 
 }  // namespace

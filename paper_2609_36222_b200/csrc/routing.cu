@@ -374,16 +374,13 @@ __global__ void __launch_bounds__(kRoutingThreads) routing_kernel(RoutingArgs a)
     }
     const uint32_t avail0 = avail;
     float m = 0.f, myv = 0.f;
-    int myid = kNone, first_id = kNone;
+    int myid = kNone;
     for (int k = 0; k < K; ++k) {
       uint32_t gk;
       int gi;
       take_best<NV>(key, avail, lane, gk, gi);
       const float bv = key_float(gk);
-      if (k == 0) {
-        m = (gi != kNone && bv > -INFINITY) ? bv : 0.f;
-        first_id = gi;
-      }
+      if (k == 0) m = (gi != kNone && bv > -INFINITY) ? bv : 0.f;
       if (lane == k) {
         myv = bv;
         myid = gi;
@@ -397,22 +394,38 @@ __global__ void __launch_bounds__(kRoutingThreads) routing_kernel(RoutingArgs a)
       qs += q[i];
     }
     const float S_t = warp_sum(qs);
+    // what a routed pair adds to its expert's score: the method's predicted removal cost (the loop the
+    // compiler sees in the common case), or one of the ablation scores
+    const int rule = a.score_rule;
+    if (rule == BASE_SCORE_PREDICTED) {
 #pragma unroll
-    for (int i = 0; i < NV; ++i) {
-      const int e = lane + 32 * i;
-      if (e < E) {
-        float c = 0.f;
-        if ((taken >> i) & 1u) {
-          const float w = S_t > 0.f ? q[i] / S_t : 0.f;
-          switch (a.score_rule) {
-            case BASE_SCORE_WEIGHT_SQ: c = w * w; break;
-            case BASE_SCORE_WEIGHT: c = w; break;
-            case BASE_SCORE_STATIC: c = w * w * expf(a.pred_b[e]); break;
-            case BASE_SCORE_TOP1_UNION: c = (e == first_id) ? 1.f : 0.f; break;
-            default: c = w * w * expf(sh[i]); break;
+      for (int i = 0; i < NV; ++i) {
+        const int e = lane + 32 * i;
+        if (e < E) {
+          float c = 0.f;
+          if ((taken >> i) & 1u) {
+            const float w = S_t > 0.f ? q[i] / S_t : 0.f;
+            c = w * w * expf(sh[i]);
           }
+          a.ws.costs[size_t(t) * E + e] = c;
         }
-        a.ws.costs[size_t(t) * E + e] = c;
+      }
+    } else {
+      const int first_id = __shfl_sync(0xffffffffu, myid, 0);   // lane k holds the k-th route
+#pragma unroll 1
+      for (int i = 0; i < NV; ++i) {
+        const int e = lane + 32 * i;
+        if (e < E) {
+          float c = 0.f;
+          if ((taken >> i) & 1u) {
+            const float w = S_t > 0.f ? q[i] / S_t : 0.f;
+            if (rule == BASE_SCORE_WEIGHT_SQ) c = w * w;
+            else if (rule == BASE_SCORE_WEIGHT) c = w;
+            else if (rule == BASE_SCORE_STATIC) c = w * w * expf(a.pred_b[e]);
+            else c = (e == first_id) ? 1.f : 0.f;
+          }
+          a.ws.costs[size_t(t) * E + e] = c;
+        }
       }
     }
     if (lane < K) {
