@@ -57,7 +57,10 @@ struct Plan {
   static constexpr int kKb = kb_per_stage(kMaxN);
   static constexpr int kTileBBytes = kMaxN * 128;                                  // per k-block
   static constexpr int kStageBytes = kKb * (kTileABytes + kTileBBytes);
-  static constexpr int kExBytes = kMaxN * 64 * 4;   // up-projection exchange buffer [token][row] fp32
+  static constexpr int kExCols = kMaxN < 64 ? kMaxN : 64;     // the up-projection exchange buffer serves 64 tokens at a time
+  static constexpr int kUpBytes = kExCols * 64 * 4;           // up values [token][row] fp32
+  static constexpr int kHsBytes = kMaxN * 64 * 2;             // finished h tile [token][row] bf16, staged for wide stores
+  static constexpr int kExBytes = kUpBytes + kHsBytes;
   static constexpr int kFixed = 1024 /*alignment slack*/ + 512 /*barriers*/;
   static constexpr int kFit = (kSmemLimit - kFixed - kExBytes) / kStageBytes;
   static constexpr int kStages = kFit < kMaxStages ? kFit : kMaxStages;
@@ -111,6 +114,7 @@ struct FfnParams {
   int steps1, steps2;   // pipeline stages per unit: ceil(d/64 / 2), ceil(kb2 / 2)
   int ksplit;           // down pass: each tile's K range (I) is split over this many units (1 or 2)
   int kb2;              // down pass: k-blocks per unit = ceil(I/64 / ksplit), even
+  long long* cycles;    // developer aid (-DBASE_FFN_CYCLES)
   int split_a;          // gate/up pass: 1 = gate and up come from two maps (two boxes per k-block)
 };
 
@@ -196,6 +200,9 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
 }
 
 // 16 consecutive fp32 columns of this thread's TMEM lane.
+// SwiGLU gate with the hardware exponential and reciprocal (relative error ~1e-6, far below bf16)
+__device__ __forceinline__ float silu_fast(float x) { return __fdividef(x, 1.0f + __expf(-x)); }
+
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
   uint32_t r[16];
   asm volatile(
@@ -207,6 +214,17 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
   for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, float (&v)[8]) {
+  uint32_t r[8];
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+               : "r"(taddr)
+               : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
 }
 
 // K-major, 128-byte swizzled operand tile: rows of 128 B, 8-row groups 1024 B apart.
@@ -268,6 +286,22 @@ __device__ __forceinline__ void red_release_add(int32_t* ptr, int v) {
   asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(ptr), "r"(v) : "memory");
 }
 
+// Developer aid: with -DBASE_FFN_CYCLES every CTA writes, per role, the SM cycles it spent waiting and
+// working into p.cycles (16 counters per CTA): producer {wait empty, issue, wait token rows, stages},
+// MMA issuer {wait full, wait accumulator, issue}, epilogue warp 2 {wait, work, units}.
+#ifdef BASE_FFN_CYCLES
+#define CYC_DECL(name) long long name = 0
+#define CYC_T0(t) const long long t = clock64()
+#define CYC_ADD(name, t) name += clock64() - t
+#define CYC_OUT(i, v) if (p.cycles) p.cycles[size_t(blockIdx.x) * 16 + (i)] = (v)
+__device__ __forceinline__ long long gtime() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return (long long)t; }
+#else
+#define CYC_DECL(name)
+#define CYC_T0(t)
+#define CYC_ADD(name, t)
+#define CYC_OUT(i, v)
+#endif
+
 template <int kMaxN, int kSplit>
 __global__ void __launch_bounds__(kThreads, 1)
 ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapSet maps2, const FfnParams p) {
@@ -279,6 +313,7 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
   unsigned char* base_ptr = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   unsigned char* stages = base_ptr;
   float* ex = reinterpret_cast<float*>(base_ptr + size_t(P::kStages) * kStageBytes);
+  __nv_bfloat16* hs = reinterpret_cast<__nv_bfloat16*>(base_ptr + size_t(P::kStages) * kStageBytes + P::kUpBytes);
   Bars* bars = reinterpret_cast<Bars*>(base_ptr + size_t(P::kStages) * kStageBytes + P::kExBytes);
   volatile int* abort_flag = &bars->abort_flag;
 
@@ -320,6 +355,8 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true, x_ready = false;
+      CYC_DECL(c_wait); CYC_DECL(c_issue); CYC_DECL(c_rows); CYC_DECL(c_n); CYC_DECL(c_rows_gu); CYC_DECL(c_units); CYC_DECL(c_t_first); CYC_DECL(c_t_gu_end);
+      CYC_T0(t_start);
       // the ticket and the decoding of the next unit are requested one unit ahead, so their memory
       // latency never stalls the weight stream
       int u_cur = atomicAdd(p.counters + kCtrTicket, 1);
@@ -327,6 +364,11 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
       while (ok && u_cur < n_units) {
         const Unit un = un_next;
         int u_next = n_units;
+#ifdef BASE_FFN_CYCLES
+        long long* rec = p.cycles + 148 * 16 + (size_t(blockIdx.x) * 24 + min(int(c_units), 23)) * 8;
+        rec[0] = un.phase * 100000 + un.seg * 100 + un.tile; rec[1] = gtime(); rec[2] = 0;
+        ++c_units;
+#endif
         const bool gu = un.phase == 1;
         const int arow = gu ? un.expert * p.I + un.tile * 64 : un.expert * p.d + un.tile * 128;
         const CUtensorMap* tm_b = gu ? &maps1.b[(un.npad >> 4) - 1] : &maps2.b[(un.npad >> 4) - 1];
@@ -338,10 +380,13 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
         const int32_t* flag = gu ? p.counters + kCtrGather : p.counters + kCtrReady + un.seg;
         const int need = gu ? n_slots + (kSplit > 1 ? int(gridDim.x) : 0) : p.tiles1;
         for (int st = 0; st < n_steps; ++st) {
+          CYC_T0(t_w);
           if (!mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1u, abort_flag)) {
             ok = false;
             break;
           }
+          CYC_ADD(c_wait, t_w);
+          CYC_T0(t_i);
           const int kb = (kSplit > 1 ? un.kb0 : 0) + st * kKbPerStage;
           const uint32_t full = smem_u32(&bars->full[stage]);
           const uint32_t sa = smem_u32(stages + size_t(stage) * kStageBytes);
@@ -365,6 +410,7 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
             tma_load_3d(sa, &maps2.a, 0, arow, kb, full);            // {elem, row, k-block}
           }
           if (!b_ready) {
+            CYC_T0(t_r);
             const long long t0 = clock64();
 #pragma unroll 1
             for (uint32_t it = 0; it < kSpinLimit; ++it) {
@@ -382,6 +428,11 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
             }
             asm volatile("fence.proxy.async;" ::: "memory");   // generic-proxy writes -> async-proxy (TMA) reads
             if (gu) x_ready = true;
+            CYC_ADD(c_rows, t_r);
+#ifdef BASE_FFN_CYCLES
+            rec[2] = clock64() - t_r;
+            if (gu) { c_rows_gu += clock64() - t_r; c_t_first = clock64() - t_start; }
+#endif
           }
           tma_load_3d(sb, tm_b, 0, un.offset, kb, full);
           if (++stage == kStages) {
@@ -389,9 +440,19 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
             phase ^= 1u;
           }
           if (st == 0 && u_next < n_units) un_next = decode_unit<kSplit>(p, u_next, n_seg);
+          CYC_ADD(c_issue, t_i);
+#ifdef BASE_FFN_CYCLES
+          ++c_n;
+#endif
         }
+#ifdef BASE_FFN_CYCLES
+        if (gu) c_t_gu_end = clock64() - t_start;
+        rec[3] = gtime();
+#endif
         u_cur = u_next;
       }
+      CYC_OUT(11, c_rows_gu); CYC_OUT(12, c_t_first); CYC_OUT(13, c_t_gu_end); CYC_OUT(14, clock64() - t_start);
+      CYC_OUT(0, c_wait); CYC_OUT(1, c_issue); CYC_OUT(2, c_rows); CYC_OUT(3, c_n);
       // end of work: one more stage that carries the stop mark
       if (ok && mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1u, abort_flag)) {
         bars->stage_unit[stage].phase = 0;
@@ -404,10 +465,15 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
     if (lane == 0) {
       int stage = 0, acc = 0;
       uint32_t phase = 0, acc_phase = 0;
+      CYC_DECL(m_full); CYC_DECL(m_acc); CYC_DECL(m_issue); CYC_DECL(m_units);
       while (true) {
+        CYC_T0(t_f);
         if (!mbar_wait(smem_u32(&bars->full[stage]), phase, abort_flag)) break;
+        CYC_ADD(m_full, t_f);
         const Unit un = bars->stage_unit[stage];
+        CYC_T0(t_a);
         if (!mbar_wait(smem_u32(&bars->acc_empty[acc]), acc_phase ^ 1u, abort_flag)) break;
+        CYC_ADD(m_acc, t_a);
         bars->acc_unit[acc] = un;
         if (un.phase == 0) {
           // pass the stop mark on to the epilogue (both arrivals of the barrier)
@@ -422,10 +488,13 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
         const uint32_t tile_b = uint32_t(un.npad * 128);
         bool ok = true;
         for (int st = 0; st < n_steps; ++st) {
+          CYC_T0(t_f2);
           if (st > 0 && !mbar_wait(smem_u32(&bars->full[stage]), phase, abort_flag)) {
             ok = false;
             break;
           }
+          CYC_ADD(m_full, t_f2);
+          CYC_T0(t_m);
           tcgen05_fence_after();
           const uint32_t sa = smem_u32(stages + size_t(stage) * kStageBytes);
           const uint32_t sb = sa + kStageABytes;
@@ -444,13 +513,19 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
             stage = 0;
             phase ^= 1u;
           }
+          CYC_ADD(m_issue, t_m);
         }
         if (!ok) break;
         umma_commit(smem_u32(&bars->acc_full[acc]));
         mbar_arrive(smem_u32(&bars->acc_full[acc]));   // releases acc_unit[acc] to the epilogue
+#ifdef BASE_FFN_CYCLES
+        p.cycles[148 * 16 + (size_t(blockIdx.x) * 24 + min(int(m_units), 23)) * 8 + 4] = gtime();
+        ++m_units;
+#endif
         acc ^= 1;
         if (acc == 0) acc_phase ^= 1u;
       }
+      CYC_OUT(4, m_full); CYC_OUT(5, m_acc); CYC_OUT(6, m_issue);
     }
     __syncwarp();
   } else {
@@ -497,70 +572,102 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
     }
     int acc = 0;
     uint32_t acc_phase = 0;
+    CYC_DECL(e_wait); CYC_DECL(e_work); CYC_DECL(e_n);
     while (true) {
       int got = 0;
+      CYC_T0(t_ew);
       if (lane == 0) got = mbar_wait(smem_u32(&bars->acc_full[acc]), acc_phase, abort_flag, 128) ? 1 : 0;
       got = __shfl_sync(0xffffffffu, got, 0);
       if (!named_and(1, 128, got != 0)) break;
+      CYC_ADD(e_wait, t_ew);
       const Unit un = bars->acc_unit[acc];
       if (un.phase == 0) break;
+      CYC_T0(t_ek);
+#ifdef BASE_FFN_CYCLES
+      if (threadIdx.x == 64) p.cycles[148 * 16 + (size_t(blockIdx.x) * 24 + min(int(e_n), 23)) * 8 + 5] = gtime();
+#endif
       tcgen05_fence_after();
       const uint32_t taddr = tmem_base + (uint32_t(q * 32) << 16) + uint32_t(acc * kAccCols);
       if (un.phase == 1) {
         const int r = (q & 1) * 32 + lane;  // row inside the 64-row slice
-        if (q >= 2) {
-          // up rows: park them in shared memory for the gate warps
-          named_sync(3, 128);  // the gate warps have finished reading the previous unit's values
-          for (int c0 = 0; c0 < un.npad; c0 += 16) {
-            float v[16];
-            tmem_ld16(taddr + c0, v);
+        // Both halves of the exchange run at once: of each round's columns the up warps park the first
+        // half for the gate warps and the gate warps park the second half for the up warps, so all four
+        // warps share the activation arithmetic. The finished bf16 tile collects in shared memory.
+        const bool is_gate = q < 2;
+        float* ex_own = ex + (is_gate ? P::kExCols * 32 : 0);
+        const float* ex_other = ex + (is_gate ? 0 : P::kExCols * 32);
+        for (int h0 = 0; h0 < un.npad; h0 += P::kExCols) {
+          const int hn = min(P::kExCols, un.npad - h0);
+          const int half = hn >> 1;
+          const int park0 = h0 + (is_gate ? half : 0), comp0 = h0 + (is_gate ? 0 : half);
+          if (h0 > 0) named_sync(3, 128);  // the values parked in the previous round have been consumed
+#pragma unroll 1
+          for (int c0 = 0; c0 < half; c0 += 8) {
+            float v[8];
+            tmem_ld8(taddr + park0 + c0, v);
 #pragma unroll
-            for (int c = 0; c < 16; ++c) ex[(c0 + c) * 64 + r] = v[c];
+            for (int c = 0; c < 8; ++c) ex_own[(c0 + c) * 64 + r] = v[c];
           }
-          tcgen05_fence_before();
-          mbar_arrive(smem_u32(&bars->acc_empty[acc]));
-          __threadfence_block();
-          named_arrive(2, 128);
-        } else {
-          named_arrive(3, 128);
-          named_sync(2, 128);  // up values are in shared memory
-          __nv_bfloat16* hrow = p.h + size_t(un.offset) * p.I + un.tile * 64 + r;
-          for (int c0 = 0; c0 < un.npad; c0 += 16) {
-            float v[16];
-            tmem_ld16(taddr + c0, v);
+          named_sync(2, 128);
+#pragma unroll 1
+          for (int c0 = 0; c0 < half; c0 += 8) {
+            float v[8];
+            tmem_ld8(taddr + comp0 + c0, v);
 #pragma unroll
-            for (int c = 0; c < 16; ++c) {
-              if (c0 + c < un.count) {
-                const float up = ex[(c0 + c) * 64 + r];
-                hrow[size_t(c0 + c) * p.I] = __float2bfloat16_rn(silu_f(v[c]) * up);
-              }
+            for (int c = 0; c < 8; c += 2) {
+              const float o0 = ex_other[(c0 + c) * 64 + r], o1 = ex_other[(c0 + c + 1) * 64 + r];
+              const float h_0 = is_gate ? silu_fast(v[c]) * o0 : silu_fast(o0) * v[c];
+              const float h_1 = is_gate ? silu_fast(v[c + 1]) * o1 : silu_fast(o1) * v[c + 1];
+              const __nv_bfloat162 pk = __floats2bfloat162_rn(h_0, h_1);
+              hs[(comp0 + c0 + c) * 64 + r] = pk.x;
+              hs[(comp0 + c0 + c + 1) * 64 + r] = pk.y;
             }
           }
-          tcgen05_fence_before();
-          mbar_arrive(smem_u32(&bars->acc_empty[acc]));
-          // publish: this tile's h rows are complete once all 64 gate threads have fenced their stores
-          __threadfence();
-          named_sync(4, 64);
-          if (q == 0 && lane == 0) red_release_add(p.counters + kCtrReady + un.seg, 1);
         }
+        tcgen05_fence_before();
+        mbar_arrive(smem_u32(&bars->acc_empty[acc]));
+#ifdef BASE_FFN_CYCLES
+        long long* r2 = p.cycles + 148 * 16 + 148 * 24 * 8 + (size_t(blockIdx.x) * 24 + min(int(e_n), 23)) * 4;
+        if (threadIdx.x == 128) r2[0] = gtime();
+#endif
+        // all four warps write the tile out, 16 bytes per thread: a token's 64 values are one 128-byte line
+        named_sync(4, 128);
+#ifdef BASE_FFN_CYCLES
+        if (threadIdx.x == 128) r2[1] = gtime();
+#endif
+        {
+          const int n16 = un.count * 8;
+          __nv_bfloat16* hdst = p.h + size_t(un.offset) * p.I + un.tile * 64;
+          for (int id = int(threadIdx.x) - 64; id < n16; id += 128) {
+            const int tok = id >> 3, part = id & 7;
+            *reinterpret_cast<uint4*>(hdst + size_t(tok) * p.I + part * 8) = *reinterpret_cast<const uint4*>(hs + tok * 64 + part * 8);
+          }
+        }
+#ifdef BASE_FFN_CYCLES
+        if (threadIdx.x == 128) r2[2] = gtime();
+#endif
+        // publish: this tile's h rows are complete once every thread has fenced its stores
+        __threadfence();
+#ifdef BASE_FFN_CYCLES
+        if (threadIdx.x == 128) r2[3] = gtime();
+#endif
+        named_sync(4, 128);
+        if (threadIdx.x == 64) red_release_add(p.counters + kCtrReady + un.seg, 1);
+#ifdef BASE_FFN_CYCLES
+        if (threadIdx.x == 64) p.cycles[148 * 16 + (size_t(blockIdx.x) * 24 + min(int(e_n), 23)) * 8 + 7] = gtime();
+#endif
       } else {
         float* yrow = p.ypair + size_t(un.offset) * p.d + un.tile * 128 + q * 32 + lane;
-        if (kSplit == 1) {
-          for (int c0 = 0; c0 < un.npad; c0 += 16) {
-            float v[16];
-            tmem_ld16(taddr + c0, v);
+        for (int c0 = 0; c0 < un.npad; c0 += 16) {
+          float v[16];
+          tmem_ld16(taddr + c0, v);
 #pragma unroll
-            for (int c = 0; c < 16; ++c)
-              if (c0 + c < un.count) yrow[size_t(c0 + c) * p.d] = v[c];
-          }
-        } else {
-          // a split tile has two contributions per element; 0 + a + b does not depend on their order
-          for (int c0 = 0; c0 < un.npad; c0 += 16) {
-            float v[16];
-            tmem_ld16(taddr + c0, v);
-#pragma unroll
-            for (int c = 0; c < 16; ++c)
-              if (c0 + c < un.count) atomicAdd(yrow + size_t(c0 + c) * p.d, v[c]);
+          for (int c = 0; c < 16; ++c) {
+            if (c0 + c < un.count) {
+              // a split tile has two contributions per element; 0 + a + b does not depend on their order
+              if (kSplit == 1) yrow[size_t(c0 + c) * p.d] = v[c];
+              else atomicAdd(yrow + size_t(c0 + c) * p.d, v[c]);
+            }
           }
         }
         tcgen05_fence_before();
@@ -568,7 +675,12 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
       }
       acc ^= 1;
       if (acc == 0) acc_phase ^= 1u;
+      CYC_ADD(e_work, t_ek);
+#ifdef BASE_FFN_CYCLES
+      ++e_n;
+#endif
     }
+    if (threadIdx.x == 64) { CYC_OUT(8, e_wait); CYC_OUT(9, e_work); CYC_OUT(10, e_n); }
   }
 
   // ---------------------------------------------------------------- teardown
@@ -767,6 +879,9 @@ cudaError_t launch_ffn_tc(const base_layer_shape& s, const base_layer_weights& w
   p.slot_token = ws.slot_token;
   p.I = s.I;
   p.d = s.d;
+#ifdef BASE_FFN_CYCLES
+  p.cycles = reinterpret_cast<long long*>(ws.x_next);   // scratch that a single-layer call does not use
+#endif
   p.tiles1 = s.I / 64;
   p.tiles2 = s.d / 128;
   p.steps1 = (s.d / kBlockK + int(kKbPerStage) - 1) / int(kKbPerStage);
