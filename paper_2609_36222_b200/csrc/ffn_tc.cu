@@ -554,7 +554,8 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
             if (j < dv) dst[j] = v[i];
           }
         }
-        __threadfence();
+        // the warp barrier orders the lanes' stores before lane 0's release, which is cumulative: one
+        // device-scope fence per row instead of one per lane
         __syncwarp();
         if (lane == 0) red_release_add(p.counters + kCtrGather, 1);
       }
@@ -566,7 +567,6 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
       float4* y4 = reinterpret_cast<float4*>(p.ypair);
       for (size_t i = size_t(blockIdx.x) * 128 + (threadIdx.x - 64); i < n4; i += size_t(gridDim.x) * 128)
         y4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-      __threadfence();
       named_sync(5, 128);
       if (threadIdx.x == 64) red_release_add(p.counters + kCtrGather, 1);
     }
@@ -646,8 +646,8 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
 #ifdef BASE_FFN_CYCLES
         if (threadIdx.x == 128) r2[2] = gtime();
 #endif
-        // publish: this tile's h rows are complete once every thread has fenced its stores
-        __threadfence();
+        // publish: the barrier orders every thread's stores before the release of thread 64, which is
+        // cumulative (a device-scope fence in each of the 128 threads costs microseconds under load)
 #ifdef BASE_FFN_CYCLES
         if (threadIdx.x == 128) r2[3] = gtime();
 #endif
