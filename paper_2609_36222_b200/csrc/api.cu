@@ -96,15 +96,16 @@ int enqueue_layer(const LayerCall& c, const Workspace& ws, cudaStream_t st, int*
     ++*launches;
   }
   mark(3, st);
+  int n_split = 1;   // partial-sum copies the down pass leaves for the combine
   if (c.opt.ffn_impl == 1) {
     e = launch_ffn_simple(s, *c.w, ws, st, launches);
   } else {
-    e = launch_ffn_tc(s, *c.w, c.hidden, ws, c.T, c.budget, st, launches);
+    e = launch_ffn_tc(s, *c.w, c.hidden, ws, c.T, c.budget, st, launches, &n_split);
   }
   if (e != cudaSuccess) return cuda_fail(e);
   mark(4, st);
 
-  e = launch_combine(ws, c.hidden, c.out, c.opt.out_is_fp32, c.x_next, c.T, s.K, s.d, st);
+  e = launch_combine(ws, c.hidden, c.out, c.opt.out_is_fp32, c.x_next, c.T, s.K, s.d, n_split, st);
   if (e != cudaSuccess) return cuda_fail(e);
   ++*launches;
   mark(5, st);

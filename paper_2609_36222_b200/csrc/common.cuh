@@ -15,6 +15,7 @@ constexpr int kMaxVals = kMaxE / kWarp;
 constexpr int kMaxK = 16;
 constexpr int kMaxT = 1024;
 constexpr int kMaxSlots = 8192;     // T*K routed pairs held in shared memory by the routing kernel
+constexpr int kMaxSplit = 2;        // the down pass may split a tile's K range over up to this many work units
 constexpr int kSegTokens = 128;     // tokens of one expert handled by one FFN work unit
 
 __device__ __forceinline__ float warp_sum(float v) {
@@ -98,10 +99,12 @@ struct Workspace {
   int32_t* seg_count;     // [max_segs]
   float* tok_m;           // [T] max logit of the token
   float* tok_S;           // [T] softmax denominator over the original top-K
-  int32_t* counters;      // [16 + max_segs]: 0 n_dispatched, 1 n_segments, 2 status, 3 total slots, 4 ticket; 16.. per-segment count of finished gate/up tiles
+  int32_t* counters;      // [16 + max_segs * kMaxSplit]: 0 n_dispatched, 1 n_segments, 2 status, 3 total slots, 4 ticket; 16.. finished gate/up tiles per (segment, K chunk of the down pass)
   __nv_bfloat16* x_sorted; // [T*K + pad, d] token inputs in expert-sorted order
   __nv_bfloat16* h;        // [T*K + pad, I] silu(gate) * up, expert-sorted
-  float* ypair;            // [T*K, d] down-projection outputs per routed pair
+  float* ypair;            // [ypair_copies][T*K, d] down-projection outputs per routed pair (one copy per K split)
+  int ypair_copies;        // partial-sum copies the buffer holds (bounds the K split of the down pass)
+  size_t ypair_stride;     // floats between two copies
   __nv_bfloat16* x_next;   // [T,d] scratch for the stack / host entry points
   size_t bytes;
 };
@@ -129,7 +132,15 @@ inline Workspace carve_workspace(void* base_ptr, const base_layer_shape& s, int 
   const int segs = max_segments(s.E, T, s.K);
   w.x_sorted = static_cast<__nv_bfloat16*>(take((TK + kRowPad) * s.d * 2, 1024));
   w.h = static_cast<__nv_bfloat16*>(take((TK + kRowPad) * s.I * 2, 1024));
-  w.ypair = static_cast<float*>(take(TK * s.d * 4, 1024));
+  // Partial sums of a split down pass live side by side. A chunk keeps at least 8 k-blocks of 64, so a
+  // short I needs fewer copies; very large token counts get fewer copies too.
+  const size_t ypair_one = align_up(TK * s.d * 4, 1024);
+  const int kb_all = s.I / 64;
+  int copies = kMaxSplit;
+  while (copies > 1 && (kb_all < 8 * copies || ypair_one * copies > (size_t(256) << 20))) copies >>= 1;
+  w.ypair_copies = copies;
+  w.ypair = static_cast<float*>(take(ypair_one * w.ypair_copies, 1024));
+  w.ypair_stride = ypair_one / 4;
   w.x_next = static_cast<__nv_bfloat16*>(take(size_t(T) * s.d * 2, 1024));
   w.logits = static_cast<float*>(take(TE * 4, 256));
   w.raw = static_cast<float*>(take(TE * 4, 256));
@@ -151,7 +162,7 @@ inline Workspace carve_workspace(void* base_ptr, const base_layer_shape& s, int 
   w.seg_count = static_cast<int32_t*>(take(size_t(segs) * 4, 256));
   w.tok_m = static_cast<float*>(take(size_t(T) * 4, 256));
   w.tok_S = static_cast<float*>(take(size_t(T) * 4, 256));
-  w.counters = static_cast<int32_t*>(take(size_t(kCtrReady + segs) * 4, 256));
+  w.counters = static_cast<int32_t*>(take(size_t(kCtrReady + segs * kMaxSplit) * 4, 256));
   w.bytes = align_up(off, 1024);
   return w;
 }
@@ -180,7 +191,7 @@ cudaError_t launch_route_scores(const void* hidden, const void* router_w, const 
 cudaError_t launch_routing(const RoutingArgs& a, cudaStream_t st);
 cudaError_t launch_gather(const void* hidden, const Workspace& ws, int T, int K, int d, cudaStream_t st);
 cudaError_t launch_combine(const Workspace& ws, const void* hidden, void* out, int out_is_fp32, void* x_next,
-                           int T, int K, int d, cudaStream_t st);
+                           int T, int K, int d, int n_split, cudaStream_t st);
 
 cudaError_t launch_ffn_simple(const base_layer_shape& s, const base_layer_weights& w, const Workspace& ws,
                               cudaStream_t st, int* launches);

@@ -112,8 +112,9 @@ struct FfnParams {
   int I, d;
   int tiles1, tiles2;   // work units per segment: I/64 gate/up tiles, d/128 down tiles
   int steps1, steps2;   // pipeline stages per unit: ceil(d/64 / 2), ceil(kb2 / 2)
-  int ksplit;           // down pass: each tile's K range (I) is split over this many units (1 or 2)
-  int kb2;              // down pass: k-blocks per unit = ceil(I/64 / ksplit), even
+  int ksplit;           // down pass: each tile's K range (I) is split over this many units (a power of two, at most kMaxSplit)
+  size_t ypair_stride;  // floats between the partial-sum copies of a split down pass
+  int kb2;              // down pass: k-blocks per unit = ceil(I/64 / ksplit), even (= gate/up tiles a unit depends on)
   long long* cycles;    // developer aid (-DBASE_FFN_CYCLES)
   int split_a;          // gate/up pass: 1 = gate and up come from two maps (two boxes per k-block)
 };
@@ -254,20 +255,25 @@ __device__ __forceinline__ bool named_and(int id, int threads, bool pred) {
   return out != 0;
 }
 
+// kSplit == 1: every down tile is one unit. kSplit > 1: the K range (I) of a down tile is cut into
+// p.ksplit chunks of p.kb2 k-blocks, one unit each, chunk-major inside a segment: the units of the
+// first chunk need only the first gate/up tiles of the segment and can start while the later ones
+// are still being computed. Every chunk writes its own partial copy of the output rows.
 template <int kSplit>
 __device__ __forceinline__ Unit decode_unit(const FfnParams& p, int u, int n_seg) {
   Unit r;
   const int u1 = n_seg * p.tiles1;
   r.phase = u < u1 ? 1 : 2;
   const int v = u < u1 ? u : u - u1;
-  const int tiles = u < u1 ? p.tiles1 : p.tiles2 * kSplit;
+  const int tiles = u < u1 ? p.tiles1 : (kSplit > 1 ? p.tiles2 * p.ksplit : p.tiles2);
   const int seg = v / tiles;
   r.seg = seg;
   r.tile = v - seg * tiles;
   r.kb0 = 0;
-  if (kSplit > 1 && u >= u1) {   // (tile, half) pairs: neighbouring units share the token rows in L2
-    r.kb0 = (r.tile % kSplit) * p.kb2;
-    r.tile /= kSplit;
+  if (kSplit > 1 && u >= u1) {
+    const int chunk = r.tile / p.tiles2;
+    r.tile -= chunk * p.tiles2;
+    r.kb0 = chunk * p.kb2;
   }
   r.expert = p.seg_expert[seg];
   r.offset = p.seg_offset[seg];
@@ -340,7 +346,7 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
   // Everything above is independent of the routing result and overlaps the previous kernels.
   pdl_wait();
   const int n_seg = p.counters[kCtrSegments];
-  const int n_units = n_seg * (p.tiles1 + p.tiles2 * kSplit);
+  const int n_units = n_seg * (p.tiles1 + p.tiles2 * (kSplit > 1 ? p.ksplit : 1));
   const int n_slots = p.counters[kCtrSlots];
   tcgen05_fence_before();
   __syncthreads();
@@ -366,7 +372,7 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
         int u_next = n_units;
 #ifdef BASE_FFN_CYCLES
         long long* rec = p.cycles + 148 * 16 + (size_t(blockIdx.x) * 24 + min(int(c_units), 23)) * 8;
-        rec[0] = un.phase * 100000 + un.seg * 100 + un.tile; rec[1] = gtime(); rec[2] = 0;
+        rec[0] = un.phase * 10000000 + un.seg * 10000 + un.tile * 10 + (un.kb0 ? un.kb0 / p.kb2 : 0); rec[1] = gtime(); rec[2] = 0;
         ++c_units;
 #endif
         const bool gu = un.phase == 1;
@@ -377,8 +383,10 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
         // The token operand of a unit is produced by other CTAs: the gathered inputs (gate/up units)
         // or the h rows of the segment (down units). Weight boxes do not depend on it and go first.
         bool b_ready = gu ? x_ready : false;
-        const int32_t* flag = gu ? p.counters + kCtrGather : p.counters + kCtrReady + un.seg;
-        const int need = gu ? n_slots + (kSplit > 1 ? int(gridDim.x) : 0) : p.tiles1;
+        // gate/up units wait for the gathered rows; a down unit for the gate/up tiles of its K chunk
+        const int32_t* flag = gu ? p.counters + kCtrGather
+                                 : p.counters + kCtrReady + (kSplit > 1 ? un.seg * p.ksplit + un.kb0 / p.kb2 : un.seg);
+        const int need = gu ? n_slots : (kSplit > 1 ? min(p.kb2, p.tiles1 - un.kb0) : p.tiles1);
         for (int st = 0; st < n_steps; ++st) {
           CYC_T0(t_w);
           if (!mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1u, abort_flag)) {
@@ -560,16 +568,6 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
         if (lane == 0) red_release_add(p.counters + kCtrGather, 1);
       }
     }
-    if (kSplit > 1) {
-      // the two halves of a split down tile add into ypair, which therefore starts from zero; every
-      // CTA clears its share and reports it through the same counter as the gather
-      const size_t n4 = size_t(n_slots) * p.d / 4;
-      float4* y4 = reinterpret_cast<float4*>(p.ypair);
-      for (size_t i = size_t(blockIdx.x) * 128 + (threadIdx.x - 64); i < n4; i += size_t(gridDim.x) * 128)
-        y4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-      named_sync(5, 128);
-      if (threadIdx.x == 64) red_release_add(p.counters + kCtrGather, 1);
-    }
     int acc = 0;
     uint32_t acc_phase = 0;
     CYC_DECL(e_wait); CYC_DECL(e_work); CYC_DECL(e_n);
@@ -652,23 +650,21 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
         if (threadIdx.x == 128) r2[3] = gtime();
 #endif
         named_sync(4, 128);
-        if (threadIdx.x == 64) red_release_add(p.counters + kCtrReady + un.seg, 1);
+        if (threadIdx.x == 64)
+          red_release_add(p.counters + kCtrReady + (kSplit > 1 ? un.seg * p.ksplit + un.tile / p.kb2 : un.seg), 1);
 #ifdef BASE_FFN_CYCLES
         if (threadIdx.x == 64) p.cycles[148 * 16 + (size_t(blockIdx.x) * 24 + min(int(e_n), 23)) * 8 + 7] = gtime();
 #endif
       } else {
-        float* yrow = p.ypair + size_t(un.offset) * p.d + un.tile * 128 + q * 32 + lane;
+        // a split tile leaves one partial row per K chunk, each in its own copy of the buffer
+        float* yrow = p.ypair + (kSplit > 1 ? size_t(un.kb0 / p.kb2) * p.ypair_stride : size_t(0)) +
+                      size_t(un.offset) * p.d + un.tile * 128 + q * 32 + lane;
         for (int c0 = 0; c0 < un.npad; c0 += 16) {
           float v[16];
           tmem_ld16(taddr + c0, v);
 #pragma unroll
-          for (int c = 0; c < 16; ++c) {
-            if (c0 + c < un.count) {
-              // a split tile has two contributions per element; 0 + a + b does not depend on their order
-              if (kSplit == 1) yrow[size_t(c0 + c) * p.d] = v[c];
-              else atomicAdd(yrow + size_t(c0 + c) * p.d, v[c]);
-            }
-          }
+          for (int c = 0; c < 16; ++c)
+            if (c0 + c < un.count) yrow[size_t(c0 + c) * p.d] = v[c];
         }
         tcgen05_fence_before();
         mbar_arrive(smem_u32(&bars->acc_empty[acc]));
@@ -839,6 +835,7 @@ cudaError_t launch_variant(const MapSet& m1, const MapSet& m2, const FfnParams& 
 
 template <int kMaxN>
 cudaError_t launch_kernel(const MapSet& m1, const MapSet& m2, const FfnParams& p, int max_units, cudaStream_t st) {
+  // the second template argument only says whether the K split is in use; its factor is p.ksplit
   return p.ksplit > 1 ? launch_variant<kMaxN, 2>(m1, m2, p, max_units, st)
                       : launch_variant<kMaxN, 1>(m1, m2, p, max_units, st);
 }
@@ -846,7 +843,7 @@ cudaError_t launch_kernel(const MapSet& m1, const MapSet& m2, const FfnParams& p
 }  // namespace
 
 cudaError_t launch_ffn_tc(const base_layer_shape& s, const base_layer_weights& w, const void* hidden,
-                          const Workspace& ws, int T, int budget, cudaStream_t st, int* launches) {
+                          const Workspace& ws, int T, int budget, cudaStream_t st, int* launches, int* n_split) {
   const uint64_t slots = uint64_t(T) * s.K + kRowPad;
   const uint64_t wrows = uint64_t(s.E) * s.I;
   MapSet m1{}, m2{};
@@ -885,11 +882,19 @@ cudaError_t launch_ffn_tc(const base_layer_shape& s, const base_layer_weights& w
   p.tiles1 = s.I / 64;
   p.tiles2 = s.d / 128;
   p.steps1 = (s.d / kBlockK + int(kKbPerStage) - 1) / int(kKbPerStage);
-  // Few experts with long down rows (d/128 tiles each) leave SMs without a down unit; split K in two then.
+  // Few experts with long down rows (d/128 tiles each) leave SMs without a down unit and make every
+  // down unit wait for the whole gate/up pass of its segment; the K range (I) is then cut into chunks
+  // of at least 8 k-blocks, as many as the workspace holds partial-sum copies for. (On Mixtral-sized
+  // experts two chunks and four measured within 2% of each other; more copies cost the combine more.)
   const int kb_all = s.I / kBlockK;
   const int expect_experts = std::min(std::min(budget, s.E), T * s.K);
-  p.ksplit = (p.tiles2 * expect_experts < sm_count() && kb_all >= 8) ? 2 : 1;
-  p.kb2 = p.ksplit == 1 ? kb_all : ((kb_all + 1) / 2 + int(kKbPerStage) - 1) / int(kKbPerStage) * int(kKbPerStage);
+  const int down_units = p.tiles2 * expect_experts;
+  int want = down_units >= 2 * sm_count() ? 1 : kMaxSplit;
+  while (want > 1 && (kb_all < 8 * want || want > ws.ypair_copies)) want >>= 1;
+  p.ksplit = want;
+  p.ypair_stride = ws.ypair_stride;
+  p.kb2 = p.ksplit == 1 ? kb_all
+                        : ((kb_all + p.ksplit - 1) / p.ksplit + int(kKbPerStage) - 1) / int(kKbPerStage) * int(kKbPerStage);
   p.steps2 = (p.kb2 + int(kKbPerStage) - 1) / int(kKbPerStage);
   const int max_units = segs * (p.tiles1 + p.tiles2 * p.ksplit);
   // No expert can receive more tokens than the batch holds, which bounds the token tile.
@@ -898,6 +903,7 @@ cudaError_t launch_ffn_tc(const base_layer_shape& s, const base_layer_weights& w
   else if (T <= 64) e = launch_kernel<64>(m1, m2, p, max_units, st);
   else e = launch_kernel<128>(m1, m2, p, max_units, st);
   *launches += 1;
+  *n_split = p.ksplit;
   return e;
 }
 

@@ -4,5 +4,5 @@
 
 namespace base {
 cudaError_t launch_ffn_tc(const base_layer_shape& s, const base_layer_weights& w, const void* hidden,
-                          const Workspace& ws, int T, int budget, cudaStream_t st, int* launches);
+                          const Workspace& ws, int T, int budget, cudaStream_t st, int* launches, int* n_split);
 }

@@ -644,7 +644,7 @@ __global__ void __launch_bounds__(kRoutingThreads) routing_kernel(RoutingArgs a)
   __syncthreads();
   RT_STAMP(8)
   if (cta == 0)
-    for (int i = threadIdx.x; i < a.max_segs; i += kRoutingThreads) a.ws.counters[kCtrReady + i] = 0;
+    for (int i = threadIdx.x; i < a.max_segs * kMaxSplit; i += kRoutingThreads) a.ws.counters[kCtrReady + i] = 0;
   for (int i = gthread; i < S; i += kAllThreads) {
     const int e = s_eids[i];
     int slot = -1;
@@ -735,12 +735,16 @@ cudaError_t launch_gather(const void* hidden, const Workspace& ws, int T, int K,
 // ------------------------------------------------------------------------------------------------
 constexpr int kCombineIters = 8;  // d <= 256 threads * 4 * 8 = 8192
 
+// A down pass split over K leaves n_split partial rows per routed pair, one in each copy of ypair;
+// the combine walks the copies in order (and the K slots in order inside each), so the sum does not
+// depend on which work unit finished first.
+template <bool kSplit>
 __global__ void __launch_bounds__(256) combine_kernel(const float* __restrict__ ypair,
                                                       const int32_t* __restrict__ token_slot,
                                                       const float* __restrict__ gates,
                                                       const __nv_bfloat16* __restrict__ hidden, void* __restrict__ out,
                                                       int out_is_fp32, __nv_bfloat16* __restrict__ x_next, int K,
-                                                      int d) {
+                                                      int d, int n_split, size_t split_stride) {
   const int t = blockIdx.x;
   __shared__ int s_slot[kMaxK];
   __shared__ float s_gate[kMaxK];
@@ -759,21 +763,25 @@ __global__ void __launch_bounds__(256) combine_kernel(const float* __restrict__ 
   for (int it = 0; it < kCombineIters; ++it) {
     const int c = (it * 256 + threadIdx.x) * 4;
     if (c >= d) break;
-    float4 v[kMaxK];
-#pragma unroll
-    for (int k = 0; k < kMaxK; ++k) {
-      const int slot = s_slot[k];
-      v[k] = slot >= 0 ? *reinterpret_cast<const float4*>(ypair + size_t(slot) * d + c) : make_float4(0.f, 0.f, 0.f, 0.f);
-    }
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 1
+    for (int sp = 0; sp < (kSplit ? n_split : 1); ++sp) {
+      const float* part = ypair + size_t(sp) * split_stride;
+      float4 v[kMaxK];
 #pragma unroll
-    for (int k = 0; k < kMaxK; ++k) {
-      if (s_slot[k] >= 0) {
-        const float g = s_gate[k];
-        acc.x = fmaf(g, v[k].x, acc.x);
-        acc.y = fmaf(g, v[k].y, acc.y);
-        acc.z = fmaf(g, v[k].z, acc.z);
-        acc.w = fmaf(g, v[k].w, acc.w);
+      for (int k = 0; k < kMaxK; ++k) {
+        const int slot = s_slot[k];
+        v[k] = slot >= 0 ? *reinterpret_cast<const float4*>(part + size_t(slot) * d + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+#pragma unroll
+      for (int k = 0; k < kMaxK; ++k) {
+        if (s_slot[k] >= 0) {
+          const float g = s_gate[k];
+          acc.x = fmaf(g, v[k].x, acc.x);
+          acc.y = fmaf(g, v[k].y, acc.y);
+          acc.z = fmaf(g, v[k].z, acc.z);
+          acc.w = fmaf(g, v[k].w, acc.w);
+        }
       }
     }
     if (out) {
@@ -820,10 +828,12 @@ __global__ void __launch_bounds__(256) combine_kernel(const float* __restrict__ 
 
 // Layer-output-only variant: one thread per four columns, the K row reads of a thread are issued
 // together and nothing is shared between threads, so the kernel is two memory round trips long.
+template <bool kSplit>
 __global__ void __launch_bounds__(256) combine_out_kernel(const float* __restrict__ ypair,
                                                           const int32_t* __restrict__ token_slot,
                                                           const float* __restrict__ gates, void* __restrict__ out,
-                                                          int out_is_fp32, int K, int d) {
+                                                          int out_is_fp32, int K, int d, int n_split,
+                                                          size_t split_stride) {
   const int t = blockIdx.x;
   const int c = (blockIdx.y * 256 + threadIdx.x) * 4;
   pdl_launch_dependents();
@@ -836,18 +846,22 @@ __global__ void __launch_bounds__(256) combine_out_kernel(const float* __restric
     slot[k] = k < K ? __ldg(token_slot + t * K + k) : -1;
     g[k] = k < K ? __ldg(gates + t * K + k) : 0.f;
   }
-  float4 v[kMaxK];
-#pragma unroll
-  for (int k = 0; k < kMaxK; ++k)
-    v[k] = slot[k] >= 0 ? *reinterpret_cast<const float4*>(ypair + size_t(slot[k]) * d + c) : make_float4(0.f, 0.f, 0.f, 0.f);
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 1
+  for (int sp = 0; sp < (kSplit ? n_split : 1); ++sp) {
+    const float* part = ypair + size_t(sp) * split_stride;
+    float4 v[kMaxK];
 #pragma unroll
-  for (int k = 0; k < kMaxK; ++k) {
-    if (slot[k] >= 0) {
-      acc.x = fmaf(g[k], v[k].x, acc.x);
-      acc.y = fmaf(g[k], v[k].y, acc.y);
-      acc.z = fmaf(g[k], v[k].z, acc.z);
-      acc.w = fmaf(g[k], v[k].w, acc.w);
+    for (int k = 0; k < kMaxK; ++k)
+      v[k] = slot[k] >= 0 ? *reinterpret_cast<const float4*>(part + size_t(slot[k]) * d + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int k = 0; k < kMaxK; ++k) {
+      if (slot[k] >= 0) {
+        acc.x = fmaf(g[k], v[k].x, acc.x);
+        acc.y = fmaf(g[k], v[k].y, acc.y);
+        acc.z = fmaf(g[k], v[k].z, acc.z);
+        acc.w = fmaf(g[k], v[k].w, acc.w);
+      }
     }
   }
   if (out_is_fp32) {
@@ -862,13 +876,23 @@ __global__ void __launch_bounds__(256) combine_out_kernel(const float* __restric
 }
 
 cudaError_t launch_combine(const Workspace& ws, const void* hidden, void* out, int out_is_fp32, void* x_next,
-                           int T, int K, int d, cudaStream_t st) {
-  if (!x_next)
-    return launch_pdl(combine_out_kernel, dim3(T, (d + 1023) / 1024), dim3(256), 0, st, 1, ws.ypair, ws.token_slot,
-                      ws.exec_gates, out, out_is_fp32, K, d);
-  return launch_pdl(combine_kernel, dim3(T), dim3(256), 0, st, 1, ws.ypair, ws.token_slot, ws.exec_gates,
-                    static_cast<const __nv_bfloat16*>(hidden), out, out_is_fp32, static_cast<__nv_bfloat16*>(x_next), K,
-                    d);
+                           int T, int K, int d, int n_split, cudaStream_t st) {
+  // the unsplit case keeps its own instantiation: the loop over partial copies costs the common path 2 us
+  const dim3 grid_out(T, (d + 1023) / 1024);
+  auto h = static_cast<const __nv_bfloat16*>(hidden);
+  auto xn = static_cast<__nv_bfloat16*>(x_next);
+  if (!x_next) {
+    if (n_split > 1)
+      return launch_pdl(combine_out_kernel<true>, grid_out, dim3(256), 0, st, 1, ws.ypair, ws.token_slot, ws.exec_gates,
+                        out, out_is_fp32, K, d, n_split, ws.ypair_stride);
+    return launch_pdl(combine_out_kernel<false>, grid_out, dim3(256), 0, st, 1, ws.ypair, ws.token_slot, ws.exec_gates,
+                      out, out_is_fp32, K, d, n_split, ws.ypair_stride);
+  }
+  if (n_split > 1)
+    return launch_pdl(combine_kernel<true>, dim3(T), dim3(256), 0, st, 1, ws.ypair, ws.token_slot, ws.exec_gates, h, out,
+                      out_is_fp32, xn, K, d, n_split, ws.ypair_stride);
+  return launch_pdl(combine_kernel<false>, dim3(T), dim3(256), 0, st, 1, ws.ypair, ws.token_slot, ws.exec_gates, h, out,
+                    out_is_fp32, xn, K, d, n_split, ws.ypair_stride);
 }
 
 }  // namespace base
