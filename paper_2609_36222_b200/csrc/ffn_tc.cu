@@ -61,11 +61,15 @@ struct Plan {
   static constexpr int kUpBytes = kExCols * 64 * 4;           // up values [token][row] fp32
   static constexpr int kHsBytes = kMaxN * 64 * 2;             // finished h tile [token][row] bf16, staged for wide stores
   static constexpr int kExBytes = kUpBytes + kHsBytes;
-  static constexpr int kFixed = 1024 /*alignment slack*/ + 512 /*barriers*/;
+  static constexpr int kFixed = 1024 /*alignment slack*/ + 768 /*barriers, unit headers, slot map*/;
   static constexpr int kFit = (kSmemLimit - kFixed - kExBytes) / kStageBytes;
   static constexpr int kStages = kFit < kMaxStages ? kFit : kMaxStages;
   static constexpr int kAccCols = kMaxN < 32 ? 32 : kMaxN;   // TMEM columns per accumulator stage
   static constexpr int kTmemCols = 2 * kAccCols;
+  // Batches of at most 64 tokens run the gate/up pass densely: every selected expert is applied to all
+  // tokens of the batch straight from the layer input (no gathered copy, nothing to wait for), and
+  // only the rows of the tokens routed to it are stored.
+  static constexpr bool kDense = kMaxN <= 64;
   static constexpr size_t kSmemBytes = size_t(kFixed) + size_t(kStages) * kStageBytes + kExBytes;
   static_assert(kStages >= 2, "need at least two stages");
 };
@@ -88,8 +92,9 @@ struct Bars {
   int abort_flag;
   Unit stage_unit[kMaxStages];  // decoded unit travelling with each stage (phase 0 = no more work)
   Unit acc_unit[2];             // unit of each accumulator stage
+  int slot_map[64];             // dense gate/up units: output row of every token of the batch (-1: not routed here)
 };
-static_assert(sizeof(Bars) <= 512, "barrier block must fit its reserved space");
+static_assert(sizeof(Bars) <= 768, "barrier block must fit its reserved space");
 
 // Tensor maps of one pass. a: weights; a2: second weight matrix when gate and up cannot share one
 // map; b[i]: token operand with a box of 16*(i+1) rows.
@@ -109,6 +114,9 @@ struct FfnParams {
   const __nv_bfloat16* hidden;   // [T,d] token inputs
   __nv_bfloat16* x_sorted;       // [rows,d] token inputs in expert-sorted order (written here)
   const int32_t* slot_token;     // [rows] token of every sorted row
+  const int32_t* exec_ids;       // [T,K] executed experts per token (-1: none)
+  const int32_t* token_slot;     // [T,K] sorted row of every executed route
+  int T, K;
   int I, d;
   int tiles1, tiles2;   // work units per segment: I/64 gate/up tiles, d/128 down tiles
   int steps1, steps2;   // pipeline stages per unit: ceil(d/64 / 2), ceil(kb2 / 2)
@@ -259,7 +267,7 @@ __device__ __forceinline__ bool named_and(int id, int threads, bool pred) {
 // p.ksplit chunks of p.kb2 k-blocks, one unit each, chunk-major inside a segment: the units of the
 // first chunk need only the first gate/up tiles of the segment and can start while the later ones
 // are still being computed. Every chunk writes its own partial copy of the output rows.
-template <int kSplit>
+template <int kSplit, bool kDense>
 __device__ __forceinline__ Unit decode_unit(const FfnParams& p, int u, int n_seg) {
   Unit r;
   const int u1 = n_seg * p.tiles1;
@@ -276,10 +284,24 @@ __device__ __forceinline__ Unit decode_unit(const FfnParams& p, int u, int n_seg
     r.kb0 = chunk * p.kb2;
   }
   r.expert = p.seg_expert[seg];
-  r.offset = p.seg_offset[seg];
-  r.count = p.seg_count[seg];
+  if (kDense && u < u1) {   // all tokens of the batch, read in place
+    r.offset = 0;
+    r.count = p.T;
+  } else {
+    r.offset = p.seg_offset[seg];
+    r.count = p.seg_count[seg];
+  }
   r.npad = (r.count + 15) & ~15;
   return r;
+}
+
+// Counter of finished gate/up tiles that a down unit waits on: one per segment (per expert in dense
+// mode, where a gate/up unit is not tied to a segment) and K chunk; kb is a k-block of the down pass,
+// which is also the index of the gate/up tile that produces it.
+template <int kSplit, bool kDense>
+__device__ __forceinline__ int ready_index(const FfnParams& p, const Unit& un, int kb) {
+  const int owner = kDense ? un.expert : un.seg;
+  return kSplit > 1 ? owner * p.ksplit + kb / p.kb2 : owner;
 }
 
 // ------------------------------------------------------------------------------------------- the kernel
@@ -366,7 +388,7 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
       // the ticket and the decoding of the next unit are requested one unit ahead, so their memory
       // latency never stalls the weight stream
       int u_cur = atomicAdd(p.counters + kCtrTicket, 1);
-      Unit un_next = decode_unit<kSplit>(p, min(u_cur, max(n_units - 1, 0)), n_seg);
+      Unit un_next = decode_unit<kSplit, P::kDense>(p, min(u_cur, max(n_units - 1, 0)), n_seg);
       while (ok && u_cur < n_units) {
         const Unit un = un_next;
         int u_next = n_units;
@@ -382,10 +404,10 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
         const int n_steps = gu ? p.steps1 : p.steps2;
         // The token operand of a unit is produced by other CTAs: the gathered inputs (gate/up units)
         // or the h rows of the segment (down units). Weight boxes do not depend on it and go first.
-        bool b_ready = gu ? x_ready : false;
+        bool b_ready = gu ? (P::kDense || x_ready) : false;
         // gate/up units wait for the gathered rows; a down unit for the gate/up tiles of its K chunk
         const int32_t* flag = gu ? p.counters + kCtrGather
-                                 : p.counters + kCtrReady + (kSplit > 1 ? un.seg * p.ksplit + un.kb0 / p.kb2 : un.seg);
+                                 : p.counters + kCtrReady + ready_index<kSplit, P::kDense>(p, un, un.kb0);
         const int need = gu ? n_slots : (kSplit > 1 ? min(p.kb2, p.tiles1 - un.kb0) : p.tiles1);
         for (int st = 0; st < n_steps; ++st) {
           CYC_T0(t_w);
@@ -447,7 +469,7 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
             stage = 0;
             phase ^= 1u;
           }
-          if (st == 0 && u_next < n_units) un_next = decode_unit<kSplit>(p, u_next, n_seg);
+          if (st == 0 && u_next < n_units) un_next = decode_unit<kSplit, P::kDense>(p, u_next, n_seg);
           CYC_ADD(c_issue, t_i);
 #ifdef BASE_FFN_CYCLES
           ++c_n;
@@ -541,8 +563,9 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
     const int q = warp & 3;  // TMEM lane quarter this warp may read
     // First job: gather the token inputs into expert-sorted order (x_sorted[row] = hidden[token of
     // row]), rows dealt round-robin over all CTAs. The weight stream is already running; only the
-    // first token box of a gate/up unit waits for the global row count.
-    {
+    // first token box of a gate/up unit waits for the global row count. (Dense batches read the layer
+    // input in place and have no such step.)
+    if (!P::kDense) {
       const int ew = warp - 2;
       const int dv = p.d >> 3;
       for (int row = blockIdx.x * 4 + ew; row < n_slots; row += gridDim.x * 4) {
@@ -588,6 +611,21 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
       const uint32_t taddr = tmem_base + (uint32_t(q * 32) << 16) + uint32_t(acc * kAccCols);
       if (un.phase == 1) {
         const int r = (q & 1) * 32 + lane;  // row inside the 64-row slice
+        // dense unit: which row of h does each token of the batch own (if it is routed to this expert)?
+        // The loads are in flight while the accumulator is processed.
+        int dense_slot = -1;
+        if (P::kDense) {
+          const int t = int(threadIdx.x) - 64;
+          if (t < p.T) {
+#pragma unroll
+            for (int k = 0; k < kMaxK; ++k) {
+              if (k < p.K) {
+                const int e = __ldg(p.exec_ids + t * p.K + k), sl = __ldg(p.token_slot + t * p.K + k);
+                if (e == un.expert) dense_slot = sl;
+              }
+            }
+          }
+        }
         // Both halves of the exchange run at once: of each round's columns the up warps park the first
         // half for the gate warps and the gate warps park the second half for the up warps, so all four
         // warps share the activation arithmetic. The finished bf16 tile collects in shared memory.
@@ -629,16 +667,19 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
         if (threadIdx.x == 128) r2[0] = gtime();
 #endif
         // all four warps write the tile out, 16 bytes per thread: a token's 64 values are one 128-byte line
+        if (P::kDense && int(threadIdx.x) - 64 < 64) bars->slot_map[threadIdx.x - 64] = dense_slot;
         named_sync(4, 128);
 #ifdef BASE_FFN_CYCLES
         if (threadIdx.x == 128) r2[1] = gtime();
 #endif
         {
           const int n16 = un.count * 8;
-          __nv_bfloat16* hdst = p.h + size_t(un.offset) * p.I + un.tile * 64;
+          __nv_bfloat16* hcol = p.h + un.tile * 64;
           for (int id = int(threadIdx.x) - 64; id < n16; id += 128) {
             const int tok = id >> 3, part = id & 7;
-            *reinterpret_cast<uint4*>(hdst + size_t(tok) * p.I + part * 8) = *reinterpret_cast<const uint4*>(hs + tok * 64 + part * 8);
+            const int row = P::kDense ? bars->slot_map[tok] : un.offset + tok;
+            if (row >= 0)
+              *reinterpret_cast<uint4*>(hcol + size_t(row) * p.I + part * 8) = *reinterpret_cast<const uint4*>(hs + tok * 64 + part * 8);
           }
         }
 #ifdef BASE_FFN_CYCLES
@@ -651,7 +692,7 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
 #endif
         named_sync(4, 128);
         if (threadIdx.x == 64)
-          red_release_add(p.counters + kCtrReady + (kSplit > 1 ? un.seg * p.ksplit + un.tile / p.kb2 : un.seg), 1);
+          red_release_add(p.counters + kCtrReady + ready_index<kSplit, P::kDense>(p, un, un.tile), 1);
 #ifdef BASE_FFN_CYCLES
         if (threadIdx.x == 64) p.cycles[148 * 16 + (size_t(blockIdx.x) * 24 + min(int(e_n), 23)) * 8 + 7] = gtime();
 #endif
@@ -858,8 +899,12 @@ cudaError_t launch_ffn_tc(const base_layer_shape& s, const base_layer_weights& w
       return cudaErrorInvalidValue;
   }
   if (!map_rows_kblocks(w.w_down, uint64_t(s.E) * s.d, s.I, 128, kKbPerStage, &m2.a)) return cudaErrorInvalidValue;
+  // dense batches (at most 64 tokens) read the gate/up token operand from the layer input itself
+  const bool dense = T <= 64;
+  const void* x_rows = dense ? hidden : static_cast<const void*>(ws.x_sorted);
+  const uint64_t n_x_rows = dense ? uint64_t(T) : slots;
   for (int i = 0; i < kNumBMaps; ++i) {
-    if (!map_rows_kblocks(ws.x_sorted, slots, s.d, 16 * (i + 1), kKbPerStage, &m1.b[i]) ||
+    if (!map_rows_kblocks(x_rows, n_x_rows, s.d, 16 * (i + 1), kKbPerStage, &m1.b[i]) ||
         !map_rows_kblocks(ws.h, slots, s.I, 16 * (i + 1), kKbPerStage, &m2.b[i]))
       return cudaErrorInvalidValue;
   }
@@ -874,6 +919,10 @@ cudaError_t launch_ffn_tc(const base_layer_shape& s, const base_layer_weights& w
   p.hidden = static_cast<const __nv_bfloat16*>(hidden);
   p.x_sorted = ws.x_sorted;
   p.slot_token = ws.slot_token;
+  p.exec_ids = ws.exec_ids;
+  p.token_slot = ws.token_slot;
+  p.T = T;
+  p.K = s.K;
   p.I = s.I;
   p.d = s.d;
 #ifdef BASE_FFN_CYCLES
