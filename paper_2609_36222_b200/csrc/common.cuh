@@ -97,9 +97,10 @@ struct Workspace {
   int32_t* seg_expert;    // [max_segs] work segments: one expert, at most kSegTokens tokens
   int32_t* seg_offset;    // [max_segs] first sorted row of the segment
   int32_t* seg_count;     // [max_segs]
+  int32_t* gu_expert;     // [E] experts of the dense gate/up pass: the early list first, late additions after it
   float* tok_m;           // [T] max logit of the token
   float* tok_S;           // [T] softmax denominator over the original top-K
-  int32_t* counters;      // [16 + max_segs * kMaxSplit]: 0 n_dispatched, 1 n_segments, 2 status, 3 total slots, 4 ticket; 16.. finished gate/up tiles per (segment, K chunk of the down pass)
+  int32_t* counters;      // [16 + max_segs * kMaxSplit]: 0 n_dispatched, 1 n_segments, 2 status, 3 total slots, 4 ticket, 5 gathered rows, 6 early list (entries + 1, 0 = not yet), 7 experts of the gate/up pass; 16.. finished gate/up tiles per (segment, K chunk of the down pass)
   __nv_bfloat16* x_sorted; // [T*K + pad, d] token inputs in expert-sorted order
   __nv_bfloat16* h;        // [T*K + pad, I] silu(gate) * up, expert-sorted
   float* ypair;            // [ypair_copies][T*K, d] down-projection outputs per routed pair (one copy per K split)
@@ -110,6 +111,7 @@ struct Workspace {
 };
 
 constexpr int kCtrDispatched = 0, kCtrSegments = 1, kCtrStatus = 2, kCtrSlots = 3, kCtrTicket = 4, kCtrGather = 5,
+              kCtrEarly = 6, kCtrGuUnits = 7,
               kCtrReady = 16;
 constexpr int kRowPad = 256;  // rows readable past the last sorted row (tile over-read stays in bounds)
 
@@ -160,6 +162,7 @@ inline Workspace carve_workspace(void* base_ptr, const base_layer_shape& s, int 
   w.seg_expert = static_cast<int32_t*>(take(size_t(segs) * 4, 256));
   w.seg_offset = static_cast<int32_t*>(take(size_t(segs) * 4, 256));
   w.seg_count = static_cast<int32_t*>(take(size_t(segs) * 4, 256));
+  w.gu_expert = static_cast<int32_t*>(take(size_t(s.E) * 4, 256));
   w.tok_m = static_cast<float*>(take(size_t(T) * 4, 256));
   w.tok_S = static_cast<float*>(take(size_t(T) * 4, 256));
   w.counters = static_cast<int32_t*>(take(size_t(kCtrReady + segs * kMaxSplit) * 4, 256));

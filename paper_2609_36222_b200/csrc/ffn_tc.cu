@@ -47,6 +47,7 @@ constexpr int kSmemLimit = 227 * 1024;      // dynamic shared memory one CTA may
 constexpr int kNumBMaps = kSegTokens / 16;  // token-tile tensor maps: box heights 16, 32, ..., 128
 constexpr uint32_t kSpinLimit = 1u << 26;
 constexpr long long kWaitCycles = 4000000000ll;   // about 2 s of SM clock
+constexpr long long kEarlyPollCycles = 400000ll;  // about 200 us: how long a producer looks for the early expert list
 
 // Shared-memory plan for work units of at most kMaxN tokens: the smaller the token tile, the more
 // weight stages fit.
@@ -108,6 +109,7 @@ struct FfnParams {
   const int32_t* seg_expert;
   const int32_t* seg_offset;
   const int32_t* seg_count;
+  const int32_t* gu_expert;   // dense gate/up pass: its experts, early list first
   int32_t* counters;
   __nv_bfloat16* h;     // gate/up pass output
   float* ypair;         // down pass output
@@ -268,9 +270,8 @@ __device__ __forceinline__ bool named_and(int id, int threads, bool pred) {
 // first chunk need only the first gate/up tiles of the segment and can start while the later ones
 // are still being computed. Every chunk writes its own partial copy of the output rows.
 template <int kSplit, bool kDense>
-__device__ __forceinline__ Unit decode_unit(const FfnParams& p, int u, int n_seg) {
+__device__ __forceinline__ Unit decode_unit(const FfnParams& p, int u, int u1) {   // u1: gate/up units of the list
   Unit r;
-  const int u1 = n_seg * p.tiles1;
   r.phase = u < u1 ? 1 : 2;
   const int v = u < u1 ? u : u - u1;
   const int tiles = u < u1 ? p.tiles1 : (kSplit > 1 ? p.tiles2 * p.ksplit : p.tiles2);
@@ -283,11 +284,12 @@ __device__ __forceinline__ Unit decode_unit(const FfnParams& p, int u, int n_seg
     r.tile -= chunk * p.tiles2;
     r.kb0 = chunk * p.kb2;
   }
-  r.expert = p.seg_expert[seg];
-  if (kDense && u < u1) {   // all tokens of the batch, read in place
+  if (kDense && u < u1) {   // the seg-th expert of the gate/up list, applied to all tokens of the batch in place
+    r.expert = p.gu_expert[seg];
     r.offset = 0;
     r.count = p.T;
   } else {
+    r.expert = p.seg_expert[seg];
     r.offset = p.seg_offset[seg];
     r.count = p.seg_count[seg];
   }
@@ -365,11 +367,16 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
     if (p.split_a) asm volatile("prefetch.tensormap [%0];" ::"l"(&maps1.a2) : "memory");
   }
   if (warp == 1) tmem_alloc(smem_u32(&bars->tmem_base), kTmemCols);
-  // Everything above is independent of the routing result and overlaps the previous kernels.
-  pdl_wait();
-  const int n_seg = p.counters[kCtrSegments];
-  const int n_units = n_seg * (p.tiles1 + p.tiles2 * (kSplit > 1 ? p.ksplit : 1));
-  const int n_slots = p.counters[kCtrSlots];
+  // Everything above is independent of the routing result and overlaps the previous kernels. A dense
+  // batch does not wait for the routing kernel to end here: its producer starts on the early expert
+  // list that the routing kernel publishes while it is still running, and every role waits for the
+  // end of that kernel only when it needs the dispatch itself.
+  const int down_units_per_seg = p.tiles2 * (kSplit > 1 ? p.ksplit : 1);
+  int n_slots = 0;
+  if (!P::kDense) {
+    pdl_wait();
+    n_slots = p.counters[kCtrSlots];
+  }
   tcgen05_fence_before();
   __syncthreads();
   tcgen05_fence_after();
@@ -387,11 +394,35 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
       CYC_T0(t_start);
       // the ticket and the decoding of the next unit are requested one unit ahead, so their memory
       // latency never stalls the weight stream
+      // u1: gate/up units of the list, n_units: all units known so far. A dense batch knows only the
+      // early gate/up units at first; the rest of the list is final when the routing kernel has ended.
+      int u1 = 0, n_units = 0;
+      bool final_known = false;
+      auto make_final = [&]() {
+        pdl_wait();
+        const int n_seg = p.counters[kCtrSegments];
+        u1 = (P::kDense ? p.counters[kCtrGuUnits] : n_seg) * p.tiles1;
+        n_units = u1 + n_seg * down_units_per_seg;
+        final_known = true;
+      };
+      if (P::kDense) {
+        int flag = 0;
+        const long long t0 = clock64();
+#pragma unroll 1
+        for (uint32_t it = 0; it < kSpinLimit; ++it) {
+          flag = ld_acquire(p.counters + kCtrEarly);
+          if (flag > 0) break;
+          __nanosleep(128);
+          if ((it & 63u) == 63u && clock64() - t0 > kEarlyPollCycles) break;
+        }
+        if (flag > 0) u1 = n_units = (flag - 1) * p.tiles1;   // else: no early list seen, wait for the final one
+      }
       int u_cur = atomicAdd(p.counters + kCtrTicket, 1);
-      Unit un_next = decode_unit<kSplit, P::kDense>(p, min(u_cur, max(n_units - 1, 0)), n_seg);
+      if (!P::kDense || u_cur >= n_units) make_final();
+      Unit un_next = decode_unit<kSplit, P::kDense>(p, min(u_cur, max(n_units - 1, 0)), u1);
       while (ok && u_cur < n_units) {
         const Unit un = un_next;
-        int u_next = n_units;
+        int u_next = 0x7fffffff;
 #ifdef BASE_FFN_CYCLES
         long long* rec = p.cycles + 148 * 16 + (size_t(blockIdx.x) * 24 + min(int(c_units), 23)) * 8;
         rec[0] = un.phase * 10000000 + un.seg * 10000 + un.tile * 10 + (un.kb0 ? un.kb0 / p.kb2 : 0); rec[1] = gtime(); rec[2] = 0;
@@ -469,7 +500,10 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
             stage = 0;
             phase ^= 1u;
           }
-          if (st == 0 && u_next < n_units) un_next = decode_unit<kSplit, P::kDense>(p, u_next, n_seg);
+          if (st == 0) {
+            if (P::kDense && !final_known && u_next >= n_units) make_final();   // past the early list
+            if (u_next < n_units) un_next = decode_unit<kSplit, P::kDense>(p, u_next, u1);
+          }
           CYC_ADD(c_issue, t_i);
 #ifdef BASE_FFN_CYCLES
           ++c_n;
@@ -561,6 +595,7 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
   } else {
     // ---------------------------------------------------------------- epilogue warps
     const int q = warp & 3;  // TMEM lane quarter this warp may read
+    if (P::kDense) pdl_wait();   // the epilogue needs the dispatch (rows of the routed tokens)
     // First job: gather the token inputs into expert-sorted order (x_sorted[row] = hidden[token of
     // row]), rows dealt round-robin over all CTAs. The weight stream is already running; only the
     // first token box of a gate/up unit waits for the global row count. (Dense batches read the layer
@@ -725,7 +760,10 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
   __syncthreads();
   tcgen05_fence_after();
   if (warp == 1) tmem_dealloc(tmem_base, kTmemCols);
-  if (threadIdx.x == 0 && bars->abort_flag) atomicOr(&p.counters[kCtrStatus], BASE_DEV_WAIT_EXPIRED);
+  if (threadIdx.x == 0 && bars->abort_flag) {
+    pdl_wait();   // the routing kernel writes the status word when it ends
+    atomicOr(&p.counters[kCtrStatus], BASE_DEV_WAIT_EXPIRED);
+  }
 }
 
 // ------------------------------------------------------------------------------------------- host side
@@ -913,6 +951,7 @@ cudaError_t launch_ffn_tc(const base_layer_shape& s, const base_layer_weights& w
   p.seg_expert = ws.seg_expert;
   p.seg_offset = ws.seg_offset;
   p.seg_count = ws.seg_count;
+  p.gu_expert = ws.gu_expert;
   p.counters = ws.counters;
   p.h = ws.h;
   p.ypair = ws.ypair;

@@ -337,8 +337,9 @@ __global__ void __launch_bounds__(kRoutingThreads) routing_kernel(RoutingArgs a)
   __shared__ float s_sc[kMaxE];
   __shared__ int32_t s_off[kMaxE + 1];
   __shared__ uint8_t s_mask[kMaxE];
-  __shared__ int32_t s_wsum[kRoutingWarps], s_wseg[kRoutingWarps];
-  __shared__ int s_status;
+  __shared__ int32_t s_wsum[kRoutingWarps], s_wseg[kRoutingWarps], s_wlate[kRoutingWarps];
+  __shared__ int s_status, s_n_early;
+  __shared__ uint8_t s_early[kMaxE];
 
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int cta = int(cluster_cta_rank());
@@ -347,8 +348,23 @@ __global__ void __launch_bounds__(kRoutingThreads) routing_kernel(RoutingArgs a)
   const int gthread = cta * kRoutingThreads + threadIdx.x;
   constexpr int kAllThreads = kClusterCtas * kRoutingThreads;
   if (threadIdx.x == 0) s_status = 0;
-  pdl_launch_dependents();
   pdl_wait();
+  // The FFN kernel that follows starts on the early expert list below while this kernel is still
+  // running, so its scheduling counters are cleared here, before it is allowed to launch: the
+  // previous FFN kernel has completed (completion is transitive through the waits), and the next one
+  // cannot start before every CTA of this kernel has passed launch_dependents.
+  if (cta == 0) {
+    for (int i = threadIdx.x; i < a.max_segs * kMaxSplit; i += kRoutingThreads) a.ws.counters[kCtrReady + i] = 0;
+    if (threadIdx.x == 0) {
+      a.ws.counters[kCtrTicket] = 0;
+      a.ws.counters[kCtrGather] = 0;
+      a.ws.counters[kCtrEarly] = 0;
+      a.ws.counters[kCtrGuUnits] = 0;
+    }
+    __threadfence();
+    __syncthreads();
+  }
+  pdl_launch_dependents();
   RT_STAMP(0)
 
   // ---- 1: original routes and predicted costs (one warp per token; a lane owns entries lane+32i)
@@ -497,6 +513,33 @@ __global__ void __launch_bounds__(kRoutingThreads) routing_kernel(RoutingArgs a)
   }
   for (int i = threadIdx.x; i < ((T + 31) >> 5) * E; i += kRoutingThreads) s_bal[i] = 0u;
   __syncthreads();
+  // Early expert list for the FFN kernel, published as soon as the selection stands: every score rule
+  // sums over routed pairs only, so a selected expert with a positive score has an original route,
+  // which it keeps, and is certain to be dispatched. (Anything this rule misses, e.g. an expert that
+  // receives only backfilled tokens or whose costs underflowed, is appended once the dispatch is known;
+  // a forced mask or a non-finite score publishes an empty list.) The FFN kernel streams these experts' gate/up weights while the rest of
+  // this kernel runs.
+  if (cta == 0) {
+    const bool eligible = !a.forced_mask && s_status == 0;
+    const int e = threadIdx.x;   // E <= kRoutingThreads
+    const bool early = eligible && e < E && s_mask[e] != 0 && s_raw[e] > 0.f;
+    const uint32_t bal = __ballot_sync(0xffffffffu, early);
+    if (lane == 0) s_wsum[warp] = __popc(bal);
+    if (e < E) s_early[e] = early;
+    __syncthreads();
+    int before = 0, total = 0;
+#pragma unroll
+    for (int w = 0; w < kRoutingWarps; ++w) {
+      const int c = s_wsum[w];
+      if (w < warp) before += c;
+      total += c;
+    }
+    if (early) a.ws.gu_expert[before + __popc(bal & ((1u << lane) - 1u))] = e;
+    if (threadIdx.x == 0) s_n_early = total;
+    __syncthreads();   // orders every thread's list entries before the release below (cumulative)
+    if (threadIdx.x == 0)
+      asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(a.ws.counters + kCtrEarly), "r"(total + 1) : "memory");
+  }
   RT_STAMP(4)
 
   // ---- ... and the restricted routes of this CTA's tokens. Original routes that are still active
@@ -591,6 +634,9 @@ __global__ void __launch_bounds__(kRoutingThreads) routing_kernel(RoutingArgs a)
     if (e < E)
       for (int ch = 0; ch < n_chunks; ++ch) c += __popc(s_bal[ch * E + e]);
     const int segs = (c + kSegTokens - 1) / kSegTokens;
+    // dispatched experts that the early list does not hold follow it, in expert order
+    const bool late = cta == 0 && e < E && c > 0 && !s_early[e];
+    const uint32_t late_bal = __ballot_sync(0xffffffffu, late);
     int incl = c, sincl = segs;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -605,15 +651,19 @@ __global__ void __launch_bounds__(kRoutingThreads) routing_kernel(RoutingArgs a)
       s_wsum[warp] = incl;
       s_wseg[warp] = sincl;
     }
+    if (lane == 0) s_wlate[warp] = __popc(late_bal);
     const int ndisp = __syncthreads_count(c > 0);
-    int run = 0, nseg = 0;
+    int run = 0, nseg = 0, late_before = 0, n_late = 0;
 #pragma unroll
     for (int w = 0; w < kRoutingWarps; ++w) {
       if (w < warp) {
         run += s_wsum[w];
         nseg += s_wseg[w];
+        late_before += s_wlate[w];
       }
+      n_late += s_wlate[w];
     }
+    if (late) a.ws.gu_expert[s_n_early + late_before + __popc(late_bal & ((1u << lane) - 1u))] = e;
     const int off = run + incl - c;
     if (e < E) {
       s_off[e] = off;
@@ -635,16 +685,13 @@ __global__ void __launch_bounds__(kRoutingThreads) routing_kernel(RoutingArgs a)
       a.ws.counters[kCtrSegments] = nseg + sincl;
       a.ws.counters[kCtrSlots] = off + c;
       a.ws.counters[kCtrStatus] = s_status;
-      a.ws.counters[kCtrTicket] = 0;
-      a.ws.counters[kCtrGather] = 0;
+      a.ws.counters[kCtrGuUnits] = s_n_early + n_late;
       if (a.dbg.n_dispatched) a.dbg.n_dispatched[0] = ndisp;
       if (a.dbg.status) a.dbg.status[0] = s_status;
     }
   }
   __syncthreads();
   RT_STAMP(8)
-  if (cta == 0)
-    for (int i = threadIdx.x; i < a.max_segs * kMaxSplit; i += kRoutingThreads) a.ws.counters[kCtrReady + i] = 0;
   for (int i = gthread; i < S; i += kAllThreads) {
     const int e = s_eids[i];
     int slot = -1;
