@@ -62,15 +62,11 @@ struct Plan {
   static constexpr int kUpBytes = kExCols * 64 * 4;           // up values [token][row] fp32
   static constexpr int kHsBytes = kMaxN * 64 * 2;             // finished h tile [token][row] bf16, staged for wide stores
   static constexpr int kExBytes = kUpBytes + kHsBytes;
-  static constexpr int kFixed = 1024 /*alignment slack*/ + 768 /*barriers, unit headers, slot map*/;
+  static constexpr int kFixed = 1024 /*alignment slack*/ + 1024 /*barriers, unit headers, slot map*/;
   static constexpr int kFit = (kSmemLimit - kFixed - kExBytes) / kStageBytes;
   static constexpr int kStages = kFit < kMaxStages ? kFit : kMaxStages;
   static constexpr int kAccCols = kMaxN < 32 ? 32 : kMaxN;   // TMEM columns per accumulator stage
   static constexpr int kTmemCols = 2 * kAccCols;
-  // Batches of at most 64 tokens run the gate/up pass densely: every selected expert is applied to all
-  // tokens of the batch straight from the layer input (no gathered copy, nothing to wait for), and
-  // only the rows of the tokens routed to it are stored.
-  static constexpr bool kDense = kMaxN <= 64;
   static constexpr size_t kSmemBytes = size_t(kFixed) + size_t(kStages) * kStageBytes + kExBytes;
   static_assert(kStages >= 2, "need at least two stages");
 };
@@ -93,9 +89,9 @@ struct Bars {
   int abort_flag;
   Unit stage_unit[kMaxStages];  // decoded unit travelling with each stage (phase 0 = no more work)
   Unit acc_unit[2];             // unit of each accumulator stage
-  int slot_map[64];             // dense gate/up units: output row of every token of the batch (-1: not routed here)
+  int slot_map[128];            // dense gate/up units: output row of every token of the batch (-1: not routed here)
 };
-static_assert(sizeof(Bars) <= 768, "barrier block must fit its reserved space");
+static_assert(sizeof(Bars) <= 1024, "barrier block must fit its reserved space");
 
 // Tensor maps of one pass. a: weights; a2: second weight matrix when gate and up cannot share one
 // map; b[i]: token operand with a box of 16*(i+1) rows.
@@ -332,7 +328,10 @@ __device__ __forceinline__ long long gtime() { unsigned long long t; asm volatil
 #define CYC_OUT(i, v)
 #endif
 
-template <int kMaxN, int kSplit>
+// kDense: batches of at most 128 tokens (one token tile) run the gate/up pass densely: every selected
+// expert is applied to all tokens of the batch straight from the layer input (no gathered copy, nothing
+// to wait for), and only the rows of the tokens routed to it are stored.
+template <int kMaxN, int kSplit, bool kDense>
 __global__ void __launch_bounds__(kThreads, 1)
 ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapSet maps2, const FfnParams p) {
   using P = Plan<kMaxN>;
@@ -373,7 +372,7 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
   // end of that kernel only when it needs the dispatch itself.
   const int down_units_per_seg = p.tiles2 * (kSplit > 1 ? p.ksplit : 1);
   int n_slots = 0;
-  if (!P::kDense) {
+  if (!kDense) {
     pdl_wait();
     n_slots = p.counters[kCtrSlots];
   }
@@ -401,11 +400,11 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
       auto make_final = [&]() {
         pdl_wait();
         const int n_seg = p.counters[kCtrSegments];
-        u1 = (P::kDense ? p.counters[kCtrGuUnits] : n_seg) * p.tiles1;
+        u1 = (kDense ? p.counters[kCtrGuUnits] : n_seg) * p.tiles1;
         n_units = u1 + n_seg * down_units_per_seg;
         final_known = true;
       };
-      if (P::kDense) {
+      if (kDense) {
         int flag = 0;
         const long long t0 = clock64();
 #pragma unroll 1
@@ -418,8 +417,8 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
         if (flag > 0) u1 = n_units = (flag - 1) * p.tiles1;   // else: no early list seen, wait for the final one
       }
       int u_cur = atomicAdd(p.counters + kCtrTicket, 1);
-      if (!P::kDense || u_cur >= n_units) make_final();
-      Unit un_next = decode_unit<kSplit, P::kDense>(p, min(u_cur, max(n_units - 1, 0)), u1);
+      if (!kDense || u_cur >= n_units) make_final();
+      Unit un_next = decode_unit<kSplit, kDense>(p, min(u_cur, max(n_units - 1, 0)), u1);
       while (ok && u_cur < n_units) {
         const Unit un = un_next;
         int u_next = 0x7fffffff;
@@ -435,10 +434,10 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
         const int n_steps = gu ? p.steps1 : p.steps2;
         // The token operand of a unit is produced by other CTAs: the gathered inputs (gate/up units)
         // or the h rows of the segment (down units). Weight boxes do not depend on it and go first.
-        bool b_ready = gu ? (P::kDense || x_ready) : false;
+        bool b_ready = gu ? (kDense || x_ready) : false;
         // gate/up units wait for the gathered rows; a down unit for the gate/up tiles of its K chunk
         const int32_t* flag = gu ? p.counters + kCtrGather
-                                 : p.counters + kCtrReady + ready_index<kSplit, P::kDense>(p, un, un.kb0);
+                                 : p.counters + kCtrReady + ready_index<kSplit, kDense>(p, un, un.kb0);
         const int need = gu ? n_slots : (kSplit > 1 ? min(p.kb2, p.tiles1 - un.kb0) : p.tiles1);
         for (int st = 0; st < n_steps; ++st) {
           CYC_T0(t_w);
@@ -501,8 +500,8 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
             phase ^= 1u;
           }
           if (st == 0) {
-            if (P::kDense && !final_known && u_next >= n_units) make_final();   // past the early list
-            if (u_next < n_units) un_next = decode_unit<kSplit, P::kDense>(p, u_next, u1);
+            if (kDense && !final_known && u_next >= n_units) make_final();   // past the early list
+            if (u_next < n_units) un_next = decode_unit<kSplit, kDense>(p, u_next, u1);
           }
           CYC_ADD(c_issue, t_i);
 #ifdef BASE_FFN_CYCLES
@@ -595,12 +594,12 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
   } else {
     // ---------------------------------------------------------------- epilogue warps
     const int q = warp & 3;  // TMEM lane quarter this warp may read
-    if (P::kDense) pdl_wait();   // the epilogue needs the dispatch (rows of the routed tokens)
+    if (kDense) pdl_wait();   // the epilogue needs the dispatch (rows of the routed tokens)
     // First job: gather the token inputs into expert-sorted order (x_sorted[row] = hidden[token of
     // row]), rows dealt round-robin over all CTAs. The weight stream is already running; only the
     // first token box of a gate/up unit waits for the global row count. (Dense batches read the layer
     // input in place and have no such step.)
-    if (!P::kDense) {
+    if (!kDense) {
       const int ew = warp - 2;
       const int dv = p.d >> 3;
       for (int row = blockIdx.x * 4 + ew; row < n_slots; row += gridDim.x * 4) {
@@ -649,7 +648,7 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
         // dense unit: which row of h does each token of the batch own (if it is routed to this expert)?
         // The loads are in flight while the accumulator is processed.
         int dense_slot = -1;
-        if (P::kDense) {
+        if (kDense) {
           const int t = int(threadIdx.x) - 64;
           if (t < p.T) {
 #pragma unroll
@@ -702,7 +701,7 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
         if (threadIdx.x == 128) r2[0] = gtime();
 #endif
         // all four warps write the tile out, 16 bytes per thread: a token's 64 values are one 128-byte line
-        if (P::kDense && int(threadIdx.x) - 64 < 64) bars->slot_map[threadIdx.x - 64] = dense_slot;
+        if (kDense) bars->slot_map[threadIdx.x - 64] = dense_slot;
         named_sync(4, 128);
 #ifdef BASE_FFN_CYCLES
         if (threadIdx.x == 128) r2[1] = gtime();
@@ -712,7 +711,7 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
           __nv_bfloat16* hcol = p.h + un.tile * 64;
           for (int id = int(threadIdx.x) - 64; id < n16; id += 128) {
             const int tok = id >> 3, part = id & 7;
-            const int row = P::kDense ? bars->slot_map[tok] : un.offset + tok;
+            const int row = kDense ? bars->slot_map[tok] : un.offset + tok;
             if (row >= 0)
               *reinterpret_cast<uint4*>(hcol + size_t(row) * p.I + part * 8) = *reinterpret_cast<const uint4*>(hs + tok * 64 + part * 8);
           }
@@ -727,7 +726,7 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
 #endif
         named_sync(4, 128);
         if (threadIdx.x == 64)
-          red_release_add(p.counters + kCtrReady + ready_index<kSplit, P::kDense>(p, un, un.tile), 1);
+          red_release_add(p.counters + kCtrReady + ready_index<kSplit, kDense>(p, un, un.tile), 1);
 #ifdef BASE_FFN_CYCLES
         if (threadIdx.x == 64) p.cycles[148 * 16 + (size_t(blockIdx.x) * 24 + min(int(e_n), 23)) * 8 + 7] = gtime();
 #endif
@@ -901,22 +900,22 @@ int sm_count() {
   return n;
 }
 
-template <int kMaxN, int kSplit>
+template <int kMaxN, int kSplit, bool kDense>
 cudaError_t launch_variant(const MapSet& m1, const MapSet& m2, const FfnParams& p, int max_units, cudaStream_t st) {
-  static cudaError_t attr = cudaFuncSetAttribute(ffn_tc_kernel<kMaxN, kSplit>,
+  static cudaError_t attr = cudaFuncSetAttribute(ffn_tc_kernel<kMaxN, kSplit, kDense>,
                                                  cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                  int(Plan<kMaxN>::kSmemBytes));
   if (attr != cudaSuccess) return attr;
   const int grid = min(sm_count(), max_units);
-  return launch_pdl(ffn_tc_kernel<kMaxN, kSplit>, dim3(grid), dim3(kThreads), Plan<kMaxN>::kSmemBytes, st, 1, m1, m2,
+  return launch_pdl(ffn_tc_kernel<kMaxN, kSplit, kDense>, dim3(grid), dim3(kThreads), Plan<kMaxN>::kSmemBytes, st, 1, m1, m2,
                     p);
 }
 
-template <int kMaxN>
+template <int kMaxN, bool kDense>
 cudaError_t launch_kernel(const MapSet& m1, const MapSet& m2, const FfnParams& p, int max_units, cudaStream_t st) {
   // the second template argument only says whether the K split is in use; its factor is p.ksplit
-  return p.ksplit > 1 ? launch_variant<kMaxN, 2>(m1, m2, p, max_units, st)
-                      : launch_variant<kMaxN, 1>(m1, m2, p, max_units, st);
+  return p.ksplit > 1 ? launch_variant<kMaxN, 2, kDense>(m1, m2, p, max_units, st)
+                      : launch_variant<kMaxN, 1, kDense>(m1, m2, p, max_units, st);
 }
 
 }  // namespace
@@ -937,8 +936,8 @@ cudaError_t launch_ffn_tc(const base_layer_shape& s, const base_layer_weights& w
       return cudaErrorInvalidValue;
   }
   if (!map_rows_kblocks(w.w_down, uint64_t(s.E) * s.d, s.I, 128, kKbPerStage, &m2.a)) return cudaErrorInvalidValue;
-  // dense batches (at most 64 tokens) read the gate/up token operand from the layer input itself
-  const bool dense = T <= 64;
+  // dense batches (at most 128 tokens, one token tile) read the gate/up token operand from the layer input itself
+  const bool dense = T <= 128;
   const void* x_rows = dense ? hidden : static_cast<const void*>(ws.x_sorted);
   const uint64_t n_x_rows = dense ? uint64_t(T) : slots;
   for (int i = 0; i < kNumBMaps; ++i) {
@@ -987,9 +986,10 @@ cudaError_t launch_ffn_tc(const base_layer_shape& s, const base_layer_weights& w
   const int max_units = segs * (p.tiles1 + p.tiles2 * p.ksplit);
   // No expert can receive more tokens than the batch holds, which bounds the token tile.
   cudaError_t e;
-  if (T <= 32) e = launch_kernel<32>(m1, m2, p, max_units, st);
-  else if (T <= 64) e = launch_kernel<64>(m1, m2, p, max_units, st);
-  else e = launch_kernel<128>(m1, m2, p, max_units, st);
+  if (T <= 32) e = launch_kernel<32, true>(m1, m2, p, max_units, st);
+  else if (T <= 64) e = launch_kernel<64, true>(m1, m2, p, max_units, st);
+  else if (dense) e = launch_kernel<128, true>(m1, m2, p, max_units, st);
+  else e = launch_kernel<128, false>(m1, m2, p, max_units, st);
   *launches += 1;
   *n_split = p.ksplit;
   return e;
