@@ -218,6 +218,28 @@ int base_moe_decode_stack(const base_layer_shape* shape, const base_layer_weight
                           void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Diagnostics of the selection quality (Eq. individual_expert_damage, Eq. energy_retained).
+ *
+ * base_true_removal_costs runs the layer with every original route executed (no budget) and writes,
+ * for each routed pair, its true contribution to the removal cost of its expert,
+ *     true_costs[t, u] = w_{t,u}^2 * ||E_u(z_t)||^2   (0 where u is not among the token's top-K),
+ * in the layout of base_predict_costs' output, so that base_aggregate_select turns it into the true
+ * scores D*_u and the oracle selection A* (top-M of D*). It is the quantity the predictor of
+ * Eq. log_energy_predictor is fitted to. Optional outputs (NULL to skip), all in route order:
+ * pair_energy[T,K] = ||E_u(z_t)||^2, topk_ids[T,K], topk_w[T,K]. Arguments, workspace and errors as
+ * for base_moe_decode_layer (same workspace size); the expert outputs are the bf16-stored h times
+ * W_down in fp32, so an energy carries the FFN's relative error (about 1e-2), not fp32's.
+ *
+ * base_energy_retained: out[0] = sum_{u in A} D*_u / sum_{u in A*} D*_u for an active mask A and the
+ * true scores D* (E <= 1024; budget is clipped to E; 0/0 is reported as 1). Sums run in expert order.
+ */
+int base_true_removal_costs(const base_layer_shape* shape, const base_layer_weights* weights, const void* hidden_bf16,
+                            const float* router_logits, int T, float* true_costs, float* pair_energy,
+                            int32_t* topk_ids, float* topk_w, void* workspace, size_t workspace_bytes, void* stream);
+int base_energy_retained(const float* true_scores, const uint8_t* active_mask, int E, int budget, float* out,
+                         void* stream);
+
+/*
  * Measurement hook (no counterpart in the paper). While an array of BASE_PROFILE_EVENTS cudaEvent_t
  * handles is set for the calling thread, every layer enqueued by that thread records them on its
  * stream: [0] before the first kernel, [1] after the router/predictor GEMV, [2] after the routing

@@ -27,7 +27,7 @@ EXPORTS = (
     "base_predict_costs", "base_aggregate_select", "base_moe_decode_layer_workspace_bytes",
     "base_moe_decode_layer", "base_moe_decode_layer_noalloc", "base_moe_decode_layer_host_workspace_bytes", "base_moe_decode_layer_host",
     "base_moe_decode_stack_workspace_bytes", "base_moe_decode_stack", "base_profile_events",
-    "base_last_launch_count",
+    "base_last_launch_count", "base_true_removal_costs", "base_energy_retained",
     "base_status_string", "base_last_cuda_error",
 )
 
@@ -84,6 +84,9 @@ def lib():
     L.base_moe_decode_stack_workspace_bytes.restype = C.c_size_t
     L.base_moe_decode_stack.argtypes = [C.POINTER(LayerShape), C.POINTER(LayerWeights), ip, vp, ip, ip, vp,
                                         C.POINTER(LayerOptions), vp, vp, C.c_size_t, vp]
+    L.base_true_removal_costs.argtypes = [C.POINTER(LayerShape), C.POINTER(LayerWeights), vp, vp, ip, vp, vp, vp, vp,
+                                          vp, C.c_size_t, vp]
+    L.base_energy_retained.argtypes = [vp, vp, ip, ip, vp, vp]
     L.base_profile_events.argtypes = [C.POINTER(C.c_void_p)]
     L.base_last_launch_count.restype = ip
     L.base_status_string.argtypes = [ip]
@@ -264,6 +267,31 @@ def base_moe_decode_stack(shape, weights_list, hidden, budget, out, workspace, n
     _check(lib().base_moe_decode_stack(C.byref(LayerShape(d, E, K, I)), arr, L, _ptr(hidden), T, budget, _ptr(out),
                                        C.byref(opt), _ptr(n_dispatched), _ptr(workspace), workspace.numel(),
                                        _stream(stream)))
+    return out
+
+
+def base_true_removal_costs(shape, weights, hidden, workspace, router_logits=None, stream=None):
+    """Returns (true_costs [T,E], pair_energy [T,K], topk_ids [T,K], topk_w [T,K]) of the unrestricted layer."""
+    d, E, K, I = shape
+    T = hidden.shape[0]
+    dev = hidden.device
+    assert hidden.dtype == torch.bfloat16 and hidden.shape[1] == d
+    true_costs = torch.empty(T, E, dtype=torch.float32, device=dev)
+    pair_energy = torch.empty(T, K, dtype=torch.float32, device=dev)
+    topk_ids = torch.empty(T, K, dtype=torch.int32, device=dev)
+    topk_w = torch.empty(T, K, dtype=torch.float32, device=dev)
+    _check(lib().base_true_removal_costs(C.byref(LayerShape(d, E, K, I)), C.byref(weights), _ptr(hidden),
+                                         _ptr(router_logits), T, _ptr(true_costs), _ptr(pair_energy), _ptr(topk_ids),
+                                         _ptr(topk_w), _ptr(workspace), workspace.numel(), _stream(stream)))
+    return true_costs, pair_energy, topk_ids, topk_w
+
+
+def base_energy_retained(true_scores, active_mask, budget, stream=None):
+    """Retained-energy ratio of an active mask against the top-`budget` of the true scores (1-element tensor)."""
+    assert true_scores.dtype == torch.float32 and active_mask.dtype == torch.uint8
+    out = torch.empty(1, dtype=torch.float32, device=true_scores.device)
+    _check(lib().base_energy_retained(_ptr(true_scores), _ptr(active_mask), true_scores.numel(), budget, _ptr(out),
+                                      _stream(stream)))
     return out
 
 

@@ -55,7 +55,7 @@ struct LayerCall {
 };
 
 // Enqueue one layer on `st` using an already carved workspace.
-int enqueue_layer(const LayerCall& c, const Workspace& ws, cudaStream_t st, int* launches) {
+int enqueue_layer(const LayerCall& c, const Workspace& ws, cudaStream_t st, int* launches, int* n_split_out = nullptr) {
   const base_layer_shape& s = *c.shape;
   cudaError_t e;
   const float* logits = c.router_logits;
@@ -109,6 +109,7 @@ int enqueue_layer(const LayerCall& c, const Workspace& ws, cudaStream_t st, int*
   if (e != cudaSuccess) return cuda_fail(e);
   ++*launches;
   mark(5, st);
+  if (n_split_out) *n_split_out = n_split;
   return BASE_OK;
 }
 
@@ -244,6 +245,46 @@ int base_moe_decode_layer_noalloc(const base_layer_shape* shape, const base_laye
   rc = enqueue_layer(c, ws, static_cast<cudaStream_t>(stream), &launches);
   if (rc == BASE_OK) g_last_launches = launches;
   return rc;
+}
+
+int base_true_removal_costs(const base_layer_shape* shape, const base_layer_weights* weights, const void* hidden_bf16,
+                            const float* router_logits, int T, float* true_costs, float* pair_energy,
+                            int32_t* topk_ids, float* topk_w, void* workspace, size_t workspace_bytes, void* stream) {
+  int rc = check_shape(shape, T);
+  if (rc != BASE_OK) return rc;
+  rc = check_layer_args(shape, weights, hidden_bf16, router_logits, T, shape->E, nullptr);
+  if (rc != BASE_OK) return rc;
+  if (!true_costs || !workspace || (reinterpret_cast<uintptr_t>(workspace) & 1023u)) return BASE_ERR_INVALID_ARG;
+  Workspace ws = carve_workspace(workspace, *shape, T);
+  if (ws.bytes > workspace_bytes) return BASE_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // every original route is executed: budget E, so the executed routes are the top-K with their weights
+  LayerCall c{};
+  c.shape = shape;
+  c.w = weights;
+  c.hidden = hidden_bf16;
+  c.router_logits = router_logits;
+  c.T = T;
+  c.budget = shape->E;
+  c.out = ws.x_next;   // the combined output is not wanted; bf16 [T,d] scratch of the stack wiring takes it
+  c.dbg.topk_ids = topk_ids;
+  c.dbg.topk_w = topk_w;
+  int launches = 0, n_split = 1;
+  rc = enqueue_layer(c, ws, st, &launches, &n_split);
+  if (rc != BASE_OK) return rc;
+  cudaError_t e = launch_pair_energy(ws, n_split, true_costs, pair_energy, T, shape->E, shape->K, shape->d, st);
+  if (e != cudaSuccess) return cuda_fail(e);
+  g_last_launches = launches + 1;
+  return BASE_OK;
+}
+
+int base_energy_retained(const float* true_scores, const uint8_t* active_mask, int E, int budget, float* out,
+                         void* stream) {
+  if (!true_scores || !active_mask || !out || E <= 0 || budget <= 0) return BASE_ERR_INVALID_ARG;
+  if (E > 1024) return BASE_ERR_UNSUPPORTED;
+  cudaError_t e = launch_energy_retained(true_scores, active_mask, E, budget < E ? budget : E, out,
+                                         static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? BASE_OK : cuda_fail(e);
 }
 
 size_t base_moe_decode_layer_host_workspace_bytes(const base_layer_shape* shape, int T_max) {

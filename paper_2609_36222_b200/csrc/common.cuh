@@ -196,6 +196,11 @@ cudaError_t launch_gather(const void* hidden, const Workspace& ws, int T, int K,
 cudaError_t launch_combine(const Workspace& ws, const void* hidden, void* out, int out_is_fp32, void* x_next,
                            int T, int K, int d, int n_split, cudaStream_t st);
 
+cudaError_t launch_pair_energy(const Workspace& ws, int n_split, float* true_costs, float* pair_energy, int T, int E,
+                               int K, int d, cudaStream_t st);
+cudaError_t launch_energy_retained(const float* scores, const uint8_t* mask, int E, int budget, float* out,
+                                   cudaStream_t st);
+
 cudaError_t launch_ffn_simple(const base_layer_shape& s, const base_layer_weights& w, const Workspace& ws,
                               cudaStream_t st, int* launches);
 
