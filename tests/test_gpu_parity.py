@@ -105,6 +105,18 @@ def test_simple_and_tensor_core_ffn_agree(layers):
     assert d <= 2e-3 * np.abs(a["got"]["y"]).max()
 
 
+@pytest.mark.parametrize("E,K,T", [(60, 4, 24), (64, 6, 48), (60, 4, 100)])
+def test_other_model_shapes(E, K, T):
+    """Expert counts and top-K of the paper's other two models (Sec. 4.1: 60 experts with K = 4 -- not a
+    multiple of 8, 16 or 32 -- and 64 experts with K = 6); d and I are stand-ins, kept small for the oracle."""
+    cfg = wl.LayerConfig(f"shape_E{E}_K{K}", d=1024, E=E, K=K, I=704, T=T, budgets=(8, 20))
+    host = HostLayer(cfg, T=T)
+    dl = device_layer_from_host(host, DEV)
+    for M in cfg.budgets + (E,):
+        check_layer(host, dl, M)
+    check_layer(host, dl, 20, gate_rule=B.GATE_RENORM, fill_rule=B.FILL_DROP)
+
+
 # ------------------------------------------------------------------------------- edge cases
 
 @pytest.mark.parametrize("T", [1, 5, 33, 130, 256])
