@@ -240,6 +240,49 @@ int base_energy_retained(const float* true_scores, const uint8_t* active_mask, i
                          void* stream);
 
 /*
+ * Offline calibration of the predictor on the device (App. Calibration Details): streaming
+ * sufficient statistics per expert over batches of calibration tokens, closed-form centred ridge,
+ * retransformation correction of the intercept. Protocol for one layer:
+ *
+ *   base_calib_reset(state)
+ *   for every batch:  base_calib_accumulate(batch, state)             -- pass 1: statistics
+ *   base_calib_solve(state, lambda)                                   -- a_u = (G_c + lambda I)^-1 q_c, b_u
+ *   for every batch:  base_calib_accumulate_correction(batch, state)  -- pass 2: sum of exp(s-hat)
+ *   base_calib_finalize(state, pred_A, pred_b)                        -- b_u += log(mean energy / mean exp(s-hat))
+ *
+ * accumulate runs the layer with every original route executed (as base_true_removal_costs), takes
+ * the target y = log(||E_u(z_t)||^2 + 1e-12) of every routed pair (Sec. 3.4) and adds the pair to its
+ * expert's statistics with the normalised input z/||z|| as features: count, sum y, sum y^2, sum of
+ * energies, first moments and cross-moment in fp64, Gram matrix in fp32 (a tensor-core contraction over
+ * the expert's tokens; inputs enter it as a bf16 head plus a bf16 remainder). Nothing per token is
+ * kept between batches. solve fits each expert independently from its own statistics; experts that
+ * saw no pair get a = 0 and, in finalize, b = log of the mean energy of all pairs. The correction
+ * sums exp(s-hat) under the unrounded fitted coefficients over the same batches (it needs the
+ * routes only, so it runs the router and the routing kernel but no expert); finalize folds the
+ * ratio-of-means correction into the intercept and rounds to the deployed precision (bf16 rows of
+ * pred_A, fp32 pred_b). weights->pred_A / pred_b must point to valid buffers during calibration
+ * (their values do not matter: without a budget the selection has no effect).
+ *
+ * `state` is a caller-owned device buffer of base_calib_state_bytes(shape) bytes, 256-byte aligned,
+ * holding in this order (each array 256-byte aligned): n, sum_y, sum_yy, sum_e, sum_p, coef_b
+ * ([E] fp64 each); sum_z, sum_yz, coef_a ([E,d] fp64 each); gram ([E,d,d] fp32); cg_iters ([E] int32).
+ * `workspace`: base_calib_workspace_bytes(shape, T_max) bytes, 1024-byte aligned. Limits: those of the
+ * layer, and d a multiple of 128, d <= 4096. Errors as for base_moe_decode_layer; 0 bytes = unsupported.
+ */
+size_t base_calib_state_bytes(const base_layer_shape* shape);
+size_t base_calib_workspace_bytes(const base_layer_shape* shape, int T_max);
+int base_calib_reset(const base_layer_shape* shape, void* state, size_t state_bytes, void* stream);
+int base_calib_accumulate(const base_layer_shape* shape, const base_layer_weights* weights, const void* hidden_bf16,
+                          const float* router_logits, int T, void* state, size_t state_bytes, void* workspace,
+                          size_t workspace_bytes, void* stream);
+int base_calib_solve(const base_layer_shape* shape, void* state, size_t state_bytes, double lambda, void* stream);
+int base_calib_accumulate_correction(const base_layer_shape* shape, const base_layer_weights* weights,
+                                     const void* hidden_bf16, const float* router_logits, int T, void* state,
+                                     size_t state_bytes, void* workspace, size_t workspace_bytes, void* stream);
+int base_calib_finalize(const base_layer_shape* shape, void* state, size_t state_bytes, void* pred_A_bf16,
+                        float* pred_b, void* stream);
+
+/*
  * Measurement hook (no counterpart in the paper). While an array of BASE_PROFILE_EVENTS cudaEvent_t
  * handles is set for the calling thread, every layer enqueued by that thread records them on its
  * stream: [0] before the first kernel, [1] after the router/predictor GEMV, [2] after the routing

@@ -28,6 +28,8 @@ EXPORTS = (
     "base_moe_decode_layer", "base_moe_decode_layer_noalloc", "base_moe_decode_layer_host_workspace_bytes", "base_moe_decode_layer_host",
     "base_moe_decode_stack_workspace_bytes", "base_moe_decode_stack", "base_profile_events",
     "base_last_launch_count", "base_true_removal_costs", "base_energy_retained",
+    "base_calib_state_bytes", "base_calib_workspace_bytes", "base_calib_reset", "base_calib_accumulate",
+    "base_calib_solve", "base_calib_accumulate_correction", "base_calib_finalize",
     "base_status_string", "base_last_cuda_error",
 )
 
@@ -87,6 +89,16 @@ def lib():
     L.base_true_removal_costs.argtypes = [C.POINTER(LayerShape), C.POINTER(LayerWeights), vp, vp, ip, vp, vp, vp, vp,
                                           vp, C.c_size_t, vp]
     L.base_energy_retained.argtypes = [vp, vp, ip, ip, vp, vp]
+    L.base_calib_state_bytes.argtypes = [C.POINTER(LayerShape)]
+    L.base_calib_state_bytes.restype = C.c_size_t
+    L.base_calib_workspace_bytes.argtypes = [C.POINTER(LayerShape), ip]
+    L.base_calib_workspace_bytes.restype = C.c_size_t
+    L.base_calib_reset.argtypes = [C.POINTER(LayerShape), vp, C.c_size_t, vp]
+    batch_args = [C.POINTER(LayerShape), C.POINTER(LayerWeights), vp, vp, ip, vp, C.c_size_t, vp, C.c_size_t, vp]
+    L.base_calib_accumulate.argtypes = batch_args
+    L.base_calib_accumulate_correction.argtypes = batch_args
+    L.base_calib_solve.argtypes = [C.POINTER(LayerShape), vp, C.c_size_t, C.c_double, vp]
+    L.base_calib_finalize.argtypes = [C.POINTER(LayerShape), vp, C.c_size_t, vp, vp, vp]
     L.base_profile_events.argtypes = [C.POINTER(C.c_void_p)]
     L.base_last_launch_count.restype = ip
     L.base_status_string.argtypes = [ip]
@@ -293,6 +305,68 @@ def base_energy_retained(true_scores, active_mask, budget, stream=None):
     _check(lib().base_energy_retained(_ptr(true_scores), _ptr(active_mask), true_scores.numel(), budget, _ptr(out),
                                       _stream(stream)))
     return out
+
+
+class Calibrator:
+    """Device-side calibration of one layer's predictor (thin wrapper over the base_calib_* entry points)."""
+
+    def __init__(self, shape, T_max, device):
+        self.shape = shape
+        d, E, K, I = shape
+        self._s = LayerShape(d, E, K, I)
+        n_state = lib().base_calib_state_bytes(C.byref(self._s))
+        n_ws = lib().base_calib_workspace_bytes(C.byref(self._s), T_max)
+        if n_state == 0 or n_ws == 0:
+            raise BaseError("unsupported shape")
+        self.state = alloc_workspace(n_state, device)
+        self.workspace = alloc_workspace(n_ws, device)
+        self.reset()
+
+    def reset(self, stream=None):
+        _check(lib().base_calib_reset(C.byref(self._s), _ptr(self.state), self.state.numel(), _stream(stream)))
+
+    def _batch(self, fn, weights, hidden, router_logits, stream):
+        assert hidden.dtype == torch.bfloat16 and hidden.shape[1] == self.shape[0]
+        _check(fn(C.byref(self._s), C.byref(weights), _ptr(hidden), _ptr(router_logits), hidden.shape[0],
+                  _ptr(self.state), self.state.numel(), _ptr(self.workspace), self.workspace.numel(), _stream(stream)))
+
+    def accumulate(self, weights, hidden, router_logits=None, stream=None):
+        self._batch(lib().base_calib_accumulate, weights, hidden, router_logits, stream)
+
+    def solve(self, lam, stream=None):
+        _check(lib().base_calib_solve(C.byref(self._s), _ptr(self.state), self.state.numel(), float(lam), _stream(stream)))
+
+    def accumulate_correction(self, weights, hidden, router_logits=None, stream=None):
+        self._batch(lib().base_calib_accumulate_correction, weights, hidden, router_logits, stream)
+
+    def finalize(self, stream=None):
+        d, E, K, I = self.shape
+        A = torch.empty(E, d, dtype=torch.bfloat16, device=self.state.device)
+        b = torch.empty(E, dtype=torch.float32, device=self.state.device)
+        _check(lib().base_calib_finalize(C.byref(self._s), _ptr(self.state), self.state.numel(), _ptr(A), _ptr(b),
+                                         _stream(stream)))
+        return A, b
+
+    def statistics(self):
+        """Views into the state buffer (layout of include/base_moe.h), for inspection."""
+        d, E, K, I = self.shape
+        out, off = {}, 0
+
+        def take(name, count, dtype, size):
+            nonlocal off
+            off = (off + 255) // 256 * 256
+            out[name] = self.state[off:off + count * size].view(dtype)
+            off += count * size
+
+        for name in ("n", "sum_y", "sum_yy", "sum_e", "sum_p", "coef_b"):
+            take(name, E, torch.float64, 8)
+        for name in ("sum_z", "sum_yz", "coef_a"):
+            take(name, E * d, torch.float64, 8)
+            out[name] = out[name].view(E, d)
+        take("gram", E * d * d, torch.float32, 4)
+        out["gram"] = out["gram"].view(E, d, d)
+        take("cg_iters", E, torch.int32, 4)
+        return out
 
 
 def last_launch_count():

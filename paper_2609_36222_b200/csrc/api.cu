@@ -4,6 +4,7 @@
 
 #include <mutex>
 
+#include "calib.cuh"
 #include "common.cuh"
 #include "ffn_tc.cuh"
 
@@ -54,8 +55,8 @@ struct LayerCall {
   void* x_next;  // stack wiring output or nullptr
 };
 
-// Enqueue one layer on `st` using an already carved workspace.
-int enqueue_layer(const LayerCall& c, const Workspace& ws, cudaStream_t st, int* launches, int* n_split_out = nullptr) {
+// Router + predictor GEMV and the routing kernel of one layer (selection, restricted routes, dispatch lists).
+int enqueue_routing(const LayerCall& c, const Workspace& ws, cudaStream_t st, int* launches) {
   const base_layer_shape& s = *c.shape;
   cudaError_t e;
   const float* logits = c.router_logits;
@@ -89,6 +90,15 @@ int enqueue_layer(const LayerCall& c, const Workspace& ws, cudaStream_t st, int*
   if (e != cudaSuccess) return cuda_fail(e);
   ++*launches;
   mark(2, st);
+  return BASE_OK;
+}
+
+// Enqueue one layer on `st` using an already carved workspace.
+int enqueue_layer(const LayerCall& c, const Workspace& ws, cudaStream_t st, int* launches, int* n_split_out = nullptr) {
+  const base_layer_shape& s = *c.shape;
+  cudaError_t e;
+  int rc = enqueue_routing(c, ws, st, launches);
+  if (rc != BASE_OK) return rc;
 
   if (c.opt.ffn_impl == 1) {
     e = launch_gather(c.hidden, ws, c.T, s.K, s.d, st);   // the streaming kernel gathers by itself
@@ -284,6 +294,103 @@ int base_energy_retained(const float* true_scores, const uint8_t* active_mask, i
   if (E > 1024) return BASE_ERR_UNSUPPORTED;
   cudaError_t e = launch_energy_retained(true_scores, active_mask, E, budget < E ? budget : E, out,
                                          static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? BASE_OK : cuda_fail(e);
+}
+
+// ---- calibration (App. Calibration Details) ---------------------------------------------------------
+size_t base_calib_state_bytes(const base_layer_shape* shape) {
+  if (check_shape(shape, 1) != BASE_OK || shape->d % 128 != 0 || shape->d > 4096) return 0;
+  return carve_calib_state(nullptr, *shape).bytes;
+}
+
+size_t base_calib_workspace_bytes(const base_layer_shape* shape, int T_max) {
+  if (check_shape(shape, T_max) != BASE_OK || shape->d % 128 != 0 || shape->d > 4096) return 0;
+  return carve_workspace(nullptr, *shape, T_max).bytes + carve_calib_scratch(nullptr, *shape, T_max).bytes;
+}
+
+static int check_calib(const base_layer_shape* shape, const void* state, size_t state_bytes) {
+  int rc = check_shape(shape, 1);
+  if (rc != BASE_OK) return rc;
+  if (shape->d % 128 != 0 || shape->d > 4096) return BASE_ERR_UNSUPPORTED;
+  if (!state || (reinterpret_cast<uintptr_t>(state) & 255u)) return BASE_ERR_INVALID_ARG;
+  if (carve_calib_state(nullptr, *shape).bytes > state_bytes) return BASE_ERR_WORKSPACE_TOO_SMALL;
+  return BASE_OK;
+}
+
+int base_calib_reset(const base_layer_shape* shape, void* state, size_t state_bytes, void* stream) {
+  int rc = check_calib(shape, state, state_bytes);
+  if (rc != BASE_OK) return rc;
+  cudaError_t e = cudaMemsetAsync(state, 0, carve_calib_state(nullptr, *shape).bytes, static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? BASE_OK : cuda_fail(e);
+}
+
+static int calib_batch(const base_layer_shape* shape, const base_layer_weights* weights, const void* hidden_bf16,
+                       const float* router_logits, int T, void* state, size_t state_bytes, void* workspace,
+                       size_t workspace_bytes, void* stream, bool correction_pass) {
+  int rc = check_calib(shape, state, state_bytes);
+  if (rc != BASE_OK) return rc;
+  rc = check_layer_args(shape, weights, hidden_bf16, router_logits, T, shape->E, nullptr);
+  if (rc != BASE_OK) return rc;
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 1023u)) return BASE_ERR_INVALID_ARG;
+  Workspace ws = carve_workspace(workspace, *shape, T);
+  CalibScratch sc = carve_calib_scratch(static_cast<char*>(workspace) + ws.bytes, *shape, T);
+  if (ws.bytes + sc.bytes > workspace_bytes) return BASE_ERR_WORKSPACE_TOO_SMALL;
+  CalibState st = carve_calib_state(state, *shape);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  LayerCall c{};
+  c.shape = shape;
+  c.w = weights;
+  c.hidden = hidden_bf16;
+  c.router_logits = router_logits;
+  c.T = T;
+  c.budget = shape->E;   // every original route is executed
+  c.out = ws.x_next;     // the combined output is not wanted
+  int launches = 0, n_split = 1;
+  cudaError_t e;
+  if (correction_pass) {
+    rc = enqueue_routing(c, ws, s, &launches);   // the correction needs the routes, not the experts
+    if (rc != BASE_OK) return rc;
+    e = launch_calib_correction(*shape, ws, st, hidden_bf16, T, s);
+    ++launches;
+  } else {
+    rc = enqueue_layer(c, ws, s, &launches, &n_split);
+    if (rc != BASE_OK) return rc;
+    e = launch_calib_accumulate(*shape, ws, sc, st, hidden_bf16, n_split, T, s, &launches);
+  }
+  if (e != cudaSuccess) return cuda_fail(e);
+  g_last_launches = launches;
+  return BASE_OK;
+}
+
+int base_calib_accumulate(const base_layer_shape* shape, const base_layer_weights* weights, const void* hidden_bf16,
+                          const float* router_logits, int T, void* state, size_t state_bytes, void* workspace,
+                          size_t workspace_bytes, void* stream) {
+  return calib_batch(shape, weights, hidden_bf16, router_logits, T, state, state_bytes, workspace, workspace_bytes,
+                     stream, false);
+}
+
+int base_calib_solve(const base_layer_shape* shape, void* state, size_t state_bytes, double lambda, void* stream) {
+  int rc = check_calib(shape, state, state_bytes);
+  if (rc != BASE_OK) return rc;
+  if (!(lambda > 0.0)) return BASE_ERR_INVALID_ARG;
+  cudaError_t e = launch_calib_solve(*shape, carve_calib_state(state, *shape), lambda, static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? BASE_OK : cuda_fail(e);
+}
+
+int base_calib_accumulate_correction(const base_layer_shape* shape, const base_layer_weights* weights,
+                                     const void* hidden_bf16, const float* router_logits, int T, void* state,
+                                     size_t state_bytes, void* workspace, size_t workspace_bytes, void* stream) {
+  return calib_batch(shape, weights, hidden_bf16, router_logits, T, state, state_bytes, workspace, workspace_bytes,
+                     stream, true);
+}
+
+int base_calib_finalize(const base_layer_shape* shape, void* state, size_t state_bytes, void* pred_A_bf16,
+                        float* pred_b, void* stream) {
+  int rc = check_calib(shape, state, state_bytes);
+  if (rc != BASE_OK) return rc;
+  if (!pred_A_bf16 || !pred_b) return BASE_ERR_INVALID_ARG;
+  cudaError_t e = launch_calib_finalize(*shape, carve_calib_state(state, *shape), pred_A_bf16, pred_b,
+                                        static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? BASE_OK : cuda_fail(e);
 }
 

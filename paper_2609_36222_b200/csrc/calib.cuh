@@ -1,0 +1,94 @@
+// Calibration state and scratch (App. Calibration Details): layout shared by the kernels and the entry points.
+#pragma once
+#include "common.cuh"
+
+namespace base {
+
+// Sufficient statistics of one layer, per expert. Vector and scalar statistics are fp64, the Gram
+// matrices fp32. The fitted coefficients live in the same buffer so that the correction pass and
+// the final rounding can find them.
+struct CalibState {
+  double* n;        // [E] routed pairs seen
+  double* sum_y;    // [E] sum of targets y = log(energy + eps)
+  double* sum_yy;   // [E] sum of y^2
+  double* sum_e;    // [E] sum of energies
+  double* sum_p;    // [E] sum of exp(s-hat) under the fitted coefficients (correction pass)
+  double* coef_b;   // [E] fitted intercept (before the correction)
+  double* sum_z;    // [E,d] sum of normalised inputs
+  double* sum_yz;   // [E,d] sum of y * normalised input
+  double* coef_a;   // [E,d] fitted coefficients
+  float* gram;      // [E,d,d] sum of zbar zbar^T
+  int32_t* iters;   // [E] conjugate-gradient iterations of the last solve (diagnostic)
+  size_t bytes;
+};
+
+inline CalibState carve_calib_state(void* base_ptr, const base_layer_shape& s) {
+  CalibState c{};
+  size_t off = 0;
+  char* b = static_cast<char*>(base_ptr);
+  auto take = [&](size_t bytes) -> void* {
+    off = align_up(off, 256);
+    void* p = b ? b + off : nullptr;
+    off += bytes;
+    return p;
+  };
+  const size_t E = size_t(s.E), d = size_t(s.d);
+  c.n = static_cast<double*>(take(E * 8));
+  c.sum_y = static_cast<double*>(take(E * 8));
+  c.sum_yy = static_cast<double*>(take(E * 8));
+  c.sum_e = static_cast<double*>(take(E * 8));
+  c.sum_p = static_cast<double*>(take(E * 8));
+  c.coef_b = static_cast<double*>(take(E * 8));
+  c.sum_z = static_cast<double*>(take(E * d * 8));
+  c.sum_yz = static_cast<double*>(take(E * d * 8));
+  c.coef_a = static_cast<double*>(take(E * d * 8));
+  c.gram = static_cast<float*>(take(E * d * d * 4));
+  c.iters = static_cast<int32_t*>(take(E * 4));
+  c.bytes = align_up(off, 1024);
+  return c;
+}
+
+// Scratch of one accumulate call, placed behind the layer workspace.
+struct CalibScratch {
+  float* row_energy;        // [T*K] energy of every sorted row
+  int32_t* koff;            // [E+1] first k-block (64 columns) of every expert's padded segment
+  __nv_bfloat16* zt_hi;     // [d, ld_cols] transposed normalised inputs, bf16 head
+  __nv_bfloat16* zt_lo;     // [d, ld_cols] remainder
+  size_t ld_cols;           // padded columns: T*K + 64 per expert, multiple of 64
+  size_t bytes;
+};
+
+inline CalibScratch carve_calib_scratch(void* base_ptr, const base_layer_shape& s, int T) {
+  CalibScratch c{};
+  size_t off = 0;
+  char* b = static_cast<char*>(base_ptr);
+  auto take = [&](size_t bytes) -> void* {
+    off = align_up(off, 1024);
+    void* p = b ? b + off : nullptr;
+    off += bytes;
+    return p;
+  };
+  const size_t TK = size_t(T) * s.K;
+  c.ld_cols = align_up(TK + 64 * size_t(s.E < int(TK) ? s.E : int(TK)), 64);
+  c.row_energy = static_cast<float*>(take(TK * 4));
+  c.koff = static_cast<int32_t*>(take(size_t(s.E + 1) * 4));
+  c.zt_hi = static_cast<__nv_bfloat16*>(take(size_t(s.d) * c.ld_cols * 2));
+  c.zt_lo = static_cast<__nv_bfloat16*>(take(size_t(s.d) * c.ld_cols * 2));
+  c.bytes = align_up(off, 1024);
+  return c;
+}
+
+// Statistics of the pairs left in the workspace by a layer run at budget E (enqueued on st).
+cudaError_t launch_calib_accumulate(const base_layer_shape& s, const Workspace& ws, const CalibScratch& sc,
+                                    const CalibState& st, const void* hidden, int n_split, int T, cudaStream_t stream,
+                                    int* launches);
+// Centred ridge solve per expert (conjugate gradients on the fp32 Gram matrix, fp64 vectors).
+cudaError_t launch_calib_solve(const base_layer_shape& s, const CalibState& st, double lambda, cudaStream_t stream);
+// Correction pass: adds sum exp(s-hat) of the routed pairs of this batch (routes must be in the workspace).
+cudaError_t launch_calib_correction(const base_layer_shape& s, const Workspace& ws, const CalibState& st,
+                                    const void* hidden, int T, cudaStream_t stream);
+// Intercept correction and rounding to the deployed precision.
+cudaError_t launch_calib_finalize(const base_layer_shape& s, const CalibState& st, void* pred_A_bf16, float* pred_b,
+                                  cudaStream_t stream);
+
+}  // namespace base

@@ -1,0 +1,183 @@
+// Gram update on tensor cores (included by calib.cu): G_u[i-block, j-block] += Zt_u[i-block] Zt_u[j-block]^T
+// over the expert's padded columns, for every expert and every pair of 128-row blocks. The operands
+// are the transposed inputs split as hi + lo (bf16 each); hi*hi + hi*lo + lo*hi is accumulated in
+// fp32 in TMEM, and the epilogue adds the tile into the fp32 Gram matrix in HBM (each tile has one
+// owner per launch, so the read-modify-write needs no atomics and the result is deterministic).
+//
+// HBM-bound: every launch reads and writes d*d*4 bytes per dispatched expert (the Gram matrices),
+// against 3 * 2 * d * d * n_u flops per expert.
+#pragma once
+
+namespace base {
+
+namespace {
+
+constexpr int kGramThreads = 192;
+constexpr int kGramStages = 3;
+constexpr int kGramTileBytes = 128 * 128;             // 128 rows x one k-block (64 bf16 = 128 B)
+constexpr int kGramStageBytes = 4 * kGramTileBytes;   // A hi, A lo, B hi, B lo
+constexpr int kGramMaxE = 512;
+
+struct GramBars {
+  unsigned long long full[kGramStages];
+  unsigned long long empty[kGramStages];
+  unsigned long long acc_full[2];
+  unsigned long long acc_empty[2];
+  uint32_t tmem_base;
+  int abort_flag;
+  int koff[kGramMaxE + 1];
+};
+constexpr size_t kGramSmem = 1024 + size_t(kGramStages) * kGramStageBytes + sizeof(GramBars);
+
+struct GramParams {
+  const int32_t* koff;   // [E+1]
+  float* gram;           // [E,d,d]
+  int32_t* counters;     // status word of the workspace
+  int E, d;
+};
+
+__global__ void __launch_bounds__(kGramThreads, 1)
+gram_tc_kernel(const __grid_constant__ CUtensorMap map_hi, const __grid_constant__ CUtensorMap map_lo,
+               const GramParams p) {
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* base_ptr = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  unsigned char* stages = base_ptr;
+  GramBars* bars = reinterpret_cast<GramBars*>(base_ptr + size_t(kGramStages) * kGramStageBytes);
+  volatile int* abort_flag = &bars->abort_flag;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  pdl_launch_dependents();
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kGramStages; ++s) {
+      mbar_init(smem_u32(&bars->full[s]), 1);
+      mbar_init(smem_u32(&bars->empty[s]), 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(smem_u32(&bars->acc_full[a]), 1);
+      mbar_init(smem_u32(&bars->acc_empty[a]), 128);
+    }
+    bars->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_hi) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_lo) : "memory");
+  }
+  if (warp == 1) tmem_alloc(smem_u32(&bars->tmem_base), 256);
+  pdl_wait();
+  for (int e = threadIdx.x; e <= p.E; e += kGramThreads) bars->koff[e] = p.koff[e];
+  tcgen05_fence_before();
+  __syncthreads();
+  tcgen05_fence_after();
+  const uint32_t tmem_base = bars->tmem_base;
+  const int nb = p.d >> 7;
+  const int n_units = p.E * nb * nb;
+
+  // every role walks the same static unit list: unit q = (expert, row block i, column block j)
+  if (warp == 0) {
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int q = blockIdx.x; ok && q < n_units; q += gridDim.x) {
+        const int u = q / (nb * nb), rem = q - u * nb * nb, i = rem / nb, j = rem - i * nb;
+        const int kb0 = bars->koff[u], nkb = bars->koff[u + 1] - kb0;
+        for (int kb = 0; kb < nkb; ++kb) {
+          if (!mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1u, abort_flag)) {
+            ok = false;
+            break;
+          }
+          const uint32_t full = smem_u32(&bars->full[stage]);
+          const uint32_t sa = smem_u32(stages + size_t(stage) * kGramStageBytes);
+          mbar_expect_tx(full, uint32_t(kGramStageBytes));
+          tma_load_3d(sa, &map_hi, 0, i * 128, kb0 + kb, full);
+          tma_load_3d(sa + kGramTileBytes, &map_lo, 0, i * 128, kb0 + kb, full);
+          tma_load_3d(sa + 2 * kGramTileBytes, &map_hi, 0, j * 128, kb0 + kb, full);
+          tma_load_3d(sa + 3 * kGramTileBytes, &map_lo, 0, j * 128, kb0 + kb, full);
+          if (++stage == kGramStages) {
+            stage = 0;
+            phase ^= 1u;
+          }
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    if (lane == 0) {
+      int stage = 0, acc = 0;
+      uint32_t phase = 0, acc_phase = 0;
+      const uint32_t idesc = make_idesc(128);
+      bool ok = true;
+      for (int q = blockIdx.x; ok && q < n_units; q += gridDim.x) {
+        const int u = q / (nb * nb);
+        const int nkb = bars->koff[u + 1] - bars->koff[u];
+        if (nkb == 0) continue;
+        if (!mbar_wait(smem_u32(&bars->acc_empty[acc]), acc_phase ^ 1u, abort_flag)) break;
+        const uint32_t d_tmem = tmem_base + uint32_t(acc * 128);
+        for (int kb = 0; kb < nkb; ++kb) {
+          if (!mbar_wait(smem_u32(&bars->full[stage]), phase, abort_flag)) {
+            ok = false;
+            break;
+          }
+          tcgen05_fence_after();
+          const uint32_t sa = smem_u32(stages + size_t(stage) * kGramStageBytes);
+          const uint64_t a_hi = make_smem_desc(sa), a_lo = make_smem_desc(sa + kGramTileBytes);
+          const uint64_t b_hi = make_smem_desc(sa + 2 * kGramTileBytes), b_lo = make_smem_desc(sa + 3 * kGramTileBytes);
+#pragma unroll
+          for (int k4 = 0; k4 < kBlockK / 16; ++k4) {
+            const uint64_t o = uint64_t(k4 * 2);
+            umma_bf16(d_tmem, a_hi + o, b_hi + o, idesc, uint32_t((kb | k4) != 0));
+            umma_bf16(d_tmem, a_hi + o, b_lo + o, idesc, 1u);
+            umma_bf16(d_tmem, a_lo + o, b_hi + o, idesc, 1u);
+          }
+          umma_commit(smem_u32(&bars->empty[stage]));
+          if (++stage == kGramStages) {
+            stage = 0;
+            phase ^= 1u;
+          }
+        }
+        if (!ok) break;
+        umma_commit(smem_u32(&bars->acc_full[acc]));
+        acc ^= 1;
+        if (acc == 0) acc_phase ^= 1u;
+      }
+    }
+    __syncwarp();
+  } else {
+    const int q4 = warp & 3;   // TMEM lane quarter of this warp
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    for (int q = blockIdx.x; q < n_units; q += gridDim.x) {
+      const int u = q / (nb * nb), rem = q - u * nb * nb, i = rem / nb, j = rem - i * nb;
+      if (bars->koff[u + 1] - bars->koff[u] == 0) continue;
+      if (!mbar_wait(smem_u32(&bars->acc_full[acc]), acc_phase, abort_flag, 64)) break;
+      tcgen05_fence_after();
+      const uint32_t taddr = tmem_base + (uint32_t(q4 * 32) << 16) + uint32_t(acc * 128);
+      float* g = p.gram + (size_t(u) * p.d + size_t(i) * 128 + q4 * 32 + lane) * p.d + size_t(j) * 128;
+      for (int c0 = 0; c0 < 128; c0 += 16) {
+        float v[16];
+        tmem_ld16(taddr + c0, v);
+#pragma unroll
+        for (int c = 0; c < 16; c += 4) {
+          float4 o = *reinterpret_cast<const float4*>(g + c0 + c);
+          o.x += v[c];
+          o.y += v[c + 1];
+          o.z += v[c + 2];
+          o.w += v[c + 3];
+          *reinterpret_cast<float4*>(g + c0 + c) = o;
+        }
+      }
+      tcgen05_fence_before();
+      mbar_arrive(smem_u32(&bars->acc_empty[acc]));
+      acc ^= 1;
+      if (acc == 0) acc_phase ^= 1u;
+    }
+  }
+
+  tcgen05_fence_before();
+  __syncthreads();
+  tcgen05_fence_after();
+  if (warp == 1) tmem_dealloc(tmem_base, 256);
+  if (threadIdx.x == 0 && bars->abort_flag) atomicOr(&p.counters[kCtrStatus], BASE_DEV_WAIT_EXPIRED);
+}
+
+}  // namespace
+
+}  // namespace base

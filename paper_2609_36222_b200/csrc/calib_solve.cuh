@@ -1,0 +1,240 @@
+// Ridge solve, correction pass, final rounding and the host-side launch sequences of the calibration
+// (included by calib.cu).
+#pragma once
+
+namespace base {
+
+namespace {
+
+constexpr int kSolveThreads = 1024;
+
+// Deterministic block-wide fp64 sum: strided partials, warp tree, then warp sums added in order.
+__device__ __forceinline__ double block_sum(double v, double* s_red) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_down_sync(0xffffffffu, v, o);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  __syncthreads();   // s_red may still be read from the previous call
+  if (lane == 0) s_red[warp] = v;
+  __syncthreads();
+  double t = 0.0;
+  for (int w = 0; w < int(blockDim.x >> 5); ++w) t += s_red[w];
+  return t;
+}
+
+// a = (G_c + lambda I)^-1 q_c and b = ybar - a . zbar_mean for one expert per CTA (Eq. of App.
+// Calibration Details), by conjugate gradients: G_c v = G v - n m (m . v) is applied without forming
+// the centred matrix. Vectors are fp64 in shared memory, the Gram matrix is read as stored (fp32).
+__global__ void __launch_bounds__(kSolveThreads) calib_solve_kernel(CalibState st, int d, double lambda, int iter_cap) {
+  extern __shared__ double s_vec[];
+  double* m = s_vec;          // mean of the inputs
+  double* x = m + d;          // solution
+  double* r = x + d;          // residual
+  double* pv = r + d;         // search direction
+  double* ap = pv + d;        // matrix times direction
+  __shared__ double s_red[32];
+  const int u = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const double n = st.n[u];
+  if (n < 1.0) {
+    for (int j = threadIdx.x; j < d; j += kSolveThreads) st.coef_a[size_t(u) * d + j] = 0.0;
+    if (threadIdx.x == 0) {
+      st.coef_b[u] = 0.0;
+      st.iters[u] = 0;
+    }
+    return;
+  }
+  const double sy = st.sum_y[u];
+  for (int j = threadIdx.x; j < d; j += kSolveThreads) {
+    const double mj = st.sum_z[size_t(u) * d + j] / n;
+    m[j] = mj;
+    x[j] = 0.0;
+    const double q = st.sum_yz[size_t(u) * d + j] - sy * mj;
+    r[j] = q;
+    pv[j] = q;
+  }
+  __syncthreads();
+  double part = 0.0;
+  for (int j = threadIdx.x; j < d; j += kSolveThreads) part += r[j] * r[j];
+  double rs = block_sum(part, s_red);
+  const double stop = 1e-24 * rs;   // relative residual 1e-12
+  const float* G = st.gram + size_t(u) * d * d;
+  const int max_iter = min(iter_cap, 2 * min(int(n), d) + 50);
+  int it = 0;
+  for (; it < max_iter && rs > stop && rs > 0.0; ++it) {
+    part = 0.0;
+    for (int j = threadIdx.x; j < d; j += kSolveThreads) part += m[j] * pv[j];
+    const double mp = block_sum(part, s_red);
+    for (int row = warp; row < d; row += kSolveThreads / 32) {
+      const float* g = G + size_t(row) * d;
+      double acc = 0.0;
+      for (int c = lane * 4; c < d; c += 128) {
+        const float4 gv = *reinterpret_cast<const float4*>(g + c);
+        acc += double(gv.x) * pv[c] + double(gv.y) * pv[c + 1] + double(gv.z) * pv[c + 2] + double(gv.w) * pv[c + 3];
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) acc += __shfl_down_sync(0xffffffffu, acc, o);
+      if (lane == 0) ap[row] = acc - n * m[row] * mp + lambda * pv[row];
+    }
+    __syncthreads();
+    part = 0.0;
+    for (int j = threadIdx.x; j < d; j += kSolveThreads) part += pv[j] * ap[j];
+    const double pap = block_sum(part, s_red);
+    const double alpha = rs / pap;
+    part = 0.0;
+    for (int j = threadIdx.x; j < d; j += kSolveThreads) {
+      x[j] += alpha * pv[j];
+      const double rj = r[j] - alpha * ap[j];
+      r[j] = rj;
+      part += rj * rj;
+    }
+    const double rs_new = block_sum(part, s_red);
+    const double beta = rs_new / rs;
+    for (int j = threadIdx.x; j < d; j += kSolveThreads) pv[j] = r[j] + beta * pv[j];
+    rs = rs_new;
+    __syncthreads();
+  }
+  part = 0.0;
+  for (int j = threadIdx.x; j < d; j += kSolveThreads) {
+    st.coef_a[size_t(u) * d + j] = x[j];
+    part += x[j] * m[j];
+  }
+  const double xm = block_sum(part, s_red);
+  if (threadIdx.x == 0) {
+    st.coef_b[u] = sy / n - xm;
+    st.iters[u] = it;
+  }
+}
+
+// Correction pass: sum over the expert's routed pairs of exp(a_u . zbar_t + b_u), pairs in row order.
+__global__ void __launch_bounds__(256) calib_correction_kernel(const __nv_bfloat16* __restrict__ hidden,
+                                                               const float* __restrict__ znorm2,
+                                                               const int32_t* __restrict__ slot_token,
+                                                               const int32_t* __restrict__ expert_offset,
+                                                               const int32_t* __restrict__ expert_count, int d,
+                                                               CalibState st) {
+  __shared__ double s_val[8];
+  pdl_launch_dependents();
+  pdl_wait();
+  const int u = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int cnt = expert_count[u], off = expert_offset[u];
+  if (cnt == 0 || st.n[u] < 1.0) return;
+  const double* a = st.coef_a + size_t(u) * d;
+  const double b = st.coef_b[u];
+  double total = 0.0;
+  for (int p0 = 0; p0 < cnt; p0 += 8) {
+    const int p = p0 + warp;
+    double acc = 0.0;
+    if (p < cnt) {
+      const int t = slot_token[off + p];
+      const float inv = inv_norm_of(znorm2, t);
+      for (int j = lane; j < d; j += 32) acc += a[j] * double(bf16_to_f32(hidden[size_t(t) * d + j]) * inv);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) acc += __shfl_down_sync(0xffffffffu, acc, o);
+    }
+    if (lane == 0) s_val[warp] = p < cnt ? exp(acc + b) : 0.0;
+    __syncthreads();
+    if (threadIdx.x == 0)
+      for (int w = 0; w < 8; ++w) total += s_val[w];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) st.sum_p[u] += total;
+}
+
+// b_u += log(mean energy / mean exp(s-hat)); coefficients rounded to the deployed precision (bf16
+// rows of A, fp32 b). Experts without a routed pair get a = 0 and the log of the mean energy of all pairs.
+__global__ void __launch_bounds__(256) calib_finalize_kernel(CalibState st, int E, int d,
+                                                             __nv_bfloat16* __restrict__ pred_A,
+                                                             float* __restrict__ pred_b) {
+  const int u = blockIdx.x;
+  const bool fitted = st.n[u] >= 1.0;
+  for (int j = threadIdx.x; j < d; j += 256)
+    pred_A[size_t(u) * d + j] = __float2bfloat16_rn(fitted ? float(st.coef_a[size_t(u) * d + j]) : 0.f);
+  if (threadIdx.x == 0) {
+    double b;
+    if (fitted) {
+      b = st.coef_b[u];
+      if (st.sum_p[u] > 0.0 && st.sum_e[u] > 0.0) b += log(st.sum_e[u] / st.sum_p[u]);
+    } else {
+      double te = 0.0, tn = 0.0;
+      for (int e = 0; e < E; ++e) {
+        te += st.sum_e[e];
+        tn += st.n[e];
+      }
+      b = (tn > 0.0 && te > 0.0) ? log(te / tn) : 0.0;
+    }
+    pred_b[u] = float(b);
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_calib_accumulate(const base_layer_shape& s, const Workspace& ws, const CalibScratch& sc,
+                                    const CalibState& st, const void* hidden, int n_split, int T, cudaStream_t stream,
+                                    int* launches) {
+  const __nv_bfloat16* hid = static_cast<const __nv_bfloat16*>(hidden);
+  const int TK = T * s.K;
+  cudaError_t e = launch_pdl(calib_offsets_kernel, dim3(1), dim3(512), 0, stream, 1,
+                             static_cast<const int32_t*>(ws.expert_count), s.E, sc.koff);
+  if (e != cudaSuccess) return e;
+  e = launch_pdl(calib_row_energy_kernel, dim3((TK + 7) / 8), dim3(256), 0, stream, 1,
+                 static_cast<const float*>(ws.ypair), n_split, ws.ypair_stride,
+                 static_cast<const int32_t*>(ws.counters), s.d, sc.row_energy);
+  if (e != cudaSuccess) return e;
+  e = launch_pdl(calib_transpose_kernel, dim3(unsigned(sc.ld_cols / 64), unsigned(s.d / 64)), dim3(256), 0, stream, 1,
+                 hid, static_cast<const float*>(ws.znorm2), static_cast<const int32_t*>(ws.slot_token),
+                 static_cast<const int32_t*>(ws.expert_offset), static_cast<const int32_t*>(ws.expert_count),
+                 static_cast<const int32_t*>(sc.koff), s.E, s.d, sc.ld_cols, sc.zt_hi, sc.zt_lo);
+  if (e != cudaSuccess) return e;
+  e = launch_pdl(calib_vector_stats_kernel, dim3(s.E, (s.d + 255) / 256), dim3(256), 0, stream, 1, hid,
+                 static_cast<const float*>(ws.znorm2), static_cast<const int32_t*>(ws.slot_token),
+                 static_cast<const int32_t*>(ws.expert_offset), static_cast<const int32_t*>(ws.expert_count),
+                 static_cast<const float*>(sc.row_energy), s.d, st);
+  if (e != cudaSuccess) return e;
+
+  CUtensorMap m_hi, m_lo;
+  if (!tc_map_rows_kblocks(sc.zt_hi, uint64_t(s.d), sc.ld_cols, 128, 1, &m_hi) ||
+      !tc_map_rows_kblocks(sc.zt_lo, uint64_t(s.d), sc.ld_cols, 128, 1, &m_lo))
+    return cudaErrorInvalidValue;
+  static cudaError_t attr = cudaFuncSetAttribute(gram_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kGramSmem));
+  if (attr != cudaSuccess) return attr;
+  GramParams gp{};
+  gp.koff = sc.koff;
+  gp.gram = st.gram;
+  gp.counters = ws.counters;
+  gp.E = s.E;
+  gp.d = s.d;
+  const int nb = s.d / 128;
+  const int grid = std::min(tc_sm_count(), s.E * nb * nb);
+  e = launch_pdl(gram_tc_kernel, dim3(grid), dim3(kGramThreads), kGramSmem, stream, 1, m_hi, m_lo, gp);
+  if (e != cudaSuccess) return e;
+  *launches += 5;
+  return cudaSuccess;
+}
+
+cudaError_t launch_calib_solve(const base_layer_shape& s, const CalibState& st, double lambda, cudaStream_t stream) {
+  const size_t smem = size_t(5) * s.d * sizeof(double);
+  static size_t set_for = 0;
+  if (smem > set_for) {
+    cudaError_t a = cudaFuncSetAttribute(calib_solve_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+    if (a != cudaSuccess) return a;
+    set_for = smem;
+  }
+  calib_solve_kernel<<<s.E, kSolveThreads, smem, stream>>>(st, s.d, lambda, 20000);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_calib_correction(const base_layer_shape& s, const Workspace& ws, const CalibState& st,
+                                    const void* hidden, int T, cudaStream_t stream) {
+  (void)T;
+  return launch_pdl(calib_correction_kernel, dim3(s.E), dim3(256), 0, stream, 1,
+                    static_cast<const __nv_bfloat16*>(hidden), static_cast<const float*>(ws.znorm2),
+                    static_cast<const int32_t*>(ws.slot_token), static_cast<const int32_t*>(ws.expert_offset),
+                    static_cast<const int32_t*>(ws.expert_count), s.d, st);
+}
+
+cudaError_t launch_calib_finalize(const base_layer_shape& s, const CalibState& st, void* pred_A_bf16, float* pred_b,
+                                  cudaStream_t stream) {
+  calib_finalize_kernel<<<s.E, 256, 0, stream>>>(st, s.E, s.d, static_cast<__nv_bfloat16*>(pred_A_bf16), pred_b);
+  return cudaGetLastError();
+}
+
+}  // namespace base

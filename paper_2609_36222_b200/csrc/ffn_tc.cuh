@@ -1,8 +1,15 @@
 // Tensor-core streaming FFN (tcgen05 + TMA) launcher.
 #pragma once
+#include <cuda.h>
+
 #include "common.cuh"
 
 namespace base {
+// [rows, cols] row-major bf16 matrix as a tensor map {64 elements, rows, k-blocks} with 128-byte swizzle and a box
+// of box_rows x box_kb k-blocks (cached by key). False if the driver refuses the encoding.
+bool tc_map_rows_kblocks(const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows, uint32_t box_kb,
+                          CUtensorMap* out);
+int tc_sm_count();
 cudaError_t launch_ffn_tc(const base_layer_shape& s, const base_layer_weights& w, const void* hidden,
                           const Workspace& ws, int T, int budget, cudaStream_t st, int* launches, int* n_split);
 }

@@ -1,0 +1,144 @@
+"""Device calibration of the predictor (App. Calibration Details) against the oracle's fit.
+
+Two comparisons. (1) Tight: the statistics and the ridge solution against fp64 NumPy on the SAME targets
+(the device's own pair energies), which pins the Gram contraction, the moments, the conjugate-gradient
+solve and the correction. (2) End to end: the deployed (A, b) against the oracle's fit_predictor, whose
+targets come from the fp64 experts; the difference is the FFN's error in the energies.
+"""
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import base_oracle as O
+from paper_2609_36222_b200 import binding as B
+from paper_2609_36222_b200 import workloads as wl
+from paper_2609_36222_b200.layer import bits_to_device
+
+from gpu_harness import device_layer_from_host
+from helpers import HostLayer
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+LAM = 1e-2
+EPS = 1e-12
+
+
+def _batches(cfg, sizes, **kw):
+    """One HostLayer per calibration batch: same weights (layer 0), different tokens (hidden stream of layer i)."""
+    base = HostLayer(cfg, T=sizes[0], **kw)
+    out = [base]
+    for i, T in enumerate(sizes[1:], start=1):
+        h = HostLayer(cfg, T=T, experts=None)
+        h.hidden_bits = wl.hidden_bits(cfg, T, 0, 100 + i)
+        out.append(h)
+    return base, out
+
+
+def _run_device(base, batches, dl, with_energies=True):
+    cfg = base.cfg
+    cal = B.Calibrator(dl.shape, max(h.T for h in batches), DEV)
+    logits, energies, routes = [], [], []
+    for h in batches:
+        lg = O.router_logits(h.z, base.router_w, base.router_bias)
+        logits.append(lg)
+        hid = bits_to_device(h.hidden_bits, DEV)
+        cal.accumulate(dl.weights, hid, router_logits=torch.from_numpy(lg).to(DEV))
+        if with_energies:
+            _, en, ids, _ = B.base_true_removal_costs(dl.shape, dl.weights, hid, dl.workspace,
+                                                      router_logits=torch.from_numpy(lg).to(DEV))
+            energies.append(en.cpu().numpy().astype(np.float64))
+            routes.append(ids.cpu().numpy())
+    cal.solve(LAM)
+    for h, lg in zip(batches, logits):
+        cal.accumulate_correction(dl.weights, bits_to_device(h.hidden_bits, DEV),
+                                  router_logits=torch.from_numpy(lg).to(DEV))
+    A, b = cal.finalize()
+    torch.cuda.synchronize()
+    return cal, logits, energies, routes, A.float().cpu().numpy().astype(np.float64), b.cpu().numpy().astype(np.float64)
+
+
+@pytest.mark.parametrize("name,sizes,alpha", [("tiny", (96, 128, 50, 110), 0.5), ("mid", (256, 200), None)])
+def test_calibration_statistics_and_solve_match_numpy(name, sizes, alpha):
+    cfg = wl.CONFIGS[name]
+    kw = {} if alpha is None else {"planted_alpha": alpha}
+    base, batches = _batches(cfg, sizes, **kw)
+    dl = device_layer_from_host(base, DEV, T_max=max(sizes))
+    cal, logits, energies, routes, A_dev, b_dev = _run_device(base, batches, dl)
+    st = {k: v.cpu().numpy() for k, v in cal.statistics().items() if k != "gram"}
+    d, E, K = cfg.d, cfg.E, cfg.K
+
+    zbar = [O.normalise(h.z) for h in batches]
+    for u in range(E):
+        rows = [np.nonzero((r == u).any(axis=1))[0] for r in routes]
+        X = np.concatenate([zb[tt] for zb, tt in zip(zbar, rows)])
+        en = np.concatenate([e[tt][r[tt] == u] for e, r, tt in zip(energies, routes, rows)])
+        assert st["n"][u] == len(X)                                      # integer work: exact
+        if len(X) == 0:
+            assert not A_dev[u].any()
+            continue
+        y = np.log(en + EPS)
+        np.testing.assert_allclose(st["sum_y"][u], y.sum(), rtol=1e-6, atol=1e-6)
+        np.testing.assert_allclose(st["sum_e"][u], en.sum(), rtol=1e-6)
+        np.testing.assert_allclose(st["sum_z"][u], X.sum(axis=0), rtol=0, atol=2e-6 * len(X) ** 0.5)
+        np.testing.assert_allclose(st["sum_yz"][u], (X * y[:, None]).sum(axis=0), rtol=0,
+                                   atol=2e-6 * np.abs(y).max() * len(X) ** 0.5)
+        # Gram on tensor cores from the hi + lo split of the fp32 features: about 16 bits of each input
+        G = cal.statistics()["gram"][u].cpu().numpy().astype(np.float64)
+        ref_G = X.T @ X
+        assert np.abs(G - ref_G).max() <= 1e-4 * np.abs(ref_G).max()
+        assert np.array_equal(G, G.T) or np.abs(G - G.T).max() <= 1e-6 * np.abs(ref_G).max()
+        # ridge on the same targets: predictions on the expert's own pairs
+        a_ref, b_ref = O.ridge_fit(X, y, LAM)
+        s_ref = X @ a_ref + b_ref
+        s_dev = X @ st["coef_a"][u] + st["coef_b"][u]
+        np.testing.assert_allclose(s_dev, s_ref, rtol=0, atol=2e-3)
+        assert 0 < st["cg_iters"][u] <= 2 * min(len(X), d) + 50
+        # correction and rounding: deployed intercept against the same formula in fp64
+        b_corr = st["coef_b"][u] + np.log(en.mean() / np.exp(s_dev).mean())
+        assert abs(b_dev[u] - b_corr) <= 1e-4 + 1e-6 * abs(b_corr)
+        np.testing.assert_allclose(A_dev[u], st["coef_a"][u], rtol=2 ** -8, atol=1e-30)   # bf16 rounding
+    fitted = st["n"] > 0
+    if not fitted.all():
+        mean_all = np.concatenate([e.ravel() for e in energies]).mean()
+        np.testing.assert_allclose(b_dev[~fitted], np.log(mean_all), rtol=1e-5)
+
+
+def test_calibration_end_to_end_matches_oracle_fit():
+    """Deployed coefficients against the oracle's fit on fp64 expert outputs (planted predictable energy)."""
+    cfg = wl.CONFIGS["tiny"]
+    sizes = (128, 128, 128, 128)
+    base, batches = _batches(cfg, sizes, planted_alpha=0.5)
+    dl = device_layer_from_host(base, DEV, T_max=max(sizes))
+    _, logits, _, _, A_dev, b_dev = _run_device(base, batches, dl, with_energies=False)
+    z = np.concatenate([h.z for h in batches])
+    lg = np.concatenate(logits)
+    A_ref, b_ref = O.fit_predictor(z, lg, base.expert_weights, cfg.K, cfg.E, lam=LAM, eps=EPS)
+    zbar = O.normalise(z)
+    _, R, _, _, _ = O.route_topk(lg, cfg.K)
+    worst = 0.0
+    for u in range(cfg.E):
+        tt = np.nonzero((R == u).any(axis=1))[0]
+        if tt.size == 0:
+            continue
+        s_dev = zbar[tt] @ A_dev[u] + b_dev[u]
+        s_ref = zbar[tt] @ A_ref[u] + b_ref[u]
+        worst = max(worst, np.abs(s_dev - s_ref).max())
+    # energies carry the FFN's relative error (about 1e-2, see test_gpu_diagnostics), the deployed rows bf16 rounding
+    assert worst <= 5e-2, worst
+    # and the fit is a real predictor on this workload: it explains most of the target's variance
+    u = int(np.argmax([(R == v).any(axis=1).sum() for v in range(cfg.E)]))
+    tt = np.nonzero((R == u).any(axis=1))[0]
+    out = O.expert_ffn(z[tt], *base.expert_weights(u))
+    y = np.log((out * out).sum(axis=1) + EPS)
+    s_dev = zbar[tt] @ A_dev[u] + b_dev[u]
+    assert 1 - ((y - s_dev) ** 2).sum() / ((y - y.mean()) ** 2).sum() > 0.5
+
+
+def test_calibration_error_codes():
+    cfg = wl.CONFIGS["tiny"]
+    with pytest.raises(B.BaseError, match="unsupported"):
+        B.Calibrator((8192, 8, 2, 128), 8, DEV)         # d above the calibration limit
+    cal = B.Calibrator((cfg.d, cfg.E, cfg.K, cfg.I), 8, DEV)
+    with pytest.raises(B.BaseError, match="invalid"):
+        cal.solve(0.0)
