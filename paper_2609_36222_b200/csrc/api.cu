@@ -350,8 +350,7 @@ static int calib_batch(const base_layer_shape* shape, const base_layer_weights* 
   if (correction_pass) {
     rc = enqueue_routing(c, ws, s, &launches);   // the correction needs the routes, not the experts
     if (rc != BASE_OK) return rc;
-    e = launch_calib_correction(*shape, ws, st, hidden_bf16, T, s);
-    ++launches;
+    e = launch_calib_correction(*shape, ws, sc, st, hidden_bf16, s, &launches);
   } else {
     rc = enqueue_layer(c, ws, s, &launches, &n_split);
     if (rc != BASE_OK) return rc;

@@ -77,6 +77,17 @@ __global__ void __launch_bounds__(256) calib_row_energy_kernel(const float* __re
   if (lane == 0) row_energy[row] = acc;
 }
 
+// Expert that owns k-block kb of the padded columns: last u with koff[u] <= kb.
+__device__ __forceinline__ int expert_of_kblock(const int32_t* koff, int E, int kb) {
+  int lo = 0, hi = E - 1;
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if (koff[mid] <= kb) lo = mid;
+    else hi = mid - 1;
+  }
+  return lo;
+}
+
 __device__ __forceinline__ float inv_norm_of(const float* znorm2, int t) {
   return 1.0f / fmaxf(sqrtf(znorm2[t]), 1e-30f);
 }
@@ -103,14 +114,7 @@ __global__ void __launch_bounds__(256) calib_transpose_kernel(const __nv_bfloat1
   pdl_wait();
   const int kb = blockIdx.x;
   if (kb >= koff[E]) return;
-  // expert of this k-block: last u with koff[u] <= kb (binary search over the offsets)
-  int lo = 0, hi = E - 1;
-  while (lo < hi) {
-    const int mid = (lo + hi + 1) >> 1;
-    if (koff[mid] <= kb) lo = mid;
-    else hi = mid - 1;
-  }
-  const int u = lo;
+  const int u = expert_of_kblock(koff, E, kb);
   const int pos0 = (kb - koff[u]) * 64, cnt = expert_count[u], off = expert_offset[u];
   if (threadIdx.x < 64) {
     const int pos = pos0 + threadIdx.x;
@@ -138,41 +142,90 @@ __global__ void __launch_bounds__(256) calib_transpose_kernel(const __nv_bfloat1
 }
 
 // ------------------------------------------------------------------------------------------------
-// Vector and scalar statistics in fp64: one CTA per (expert, 256 features); the expert's pairs are
-// taken in row order, so every sum has a fixed order. Thread 0 of the first feature block also
-// updates the scalars: n, sum y, sum y^2, sum energy.
+// Vector and scalar statistics in fp64, in two levels so that a popular expert (thousands of pairs
+// under a skewed router) does not serialise the pass: one CTA per (k-block of 64 pairs, 256
+// features) sums its pairs in row order into a partial; one CTA per (expert, 256 features) then adds
+// the expert's partials in k-block order to the state. Every sum has a fixed order.
 // ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) calib_vector_stats_kernel(const __nv_bfloat16* __restrict__ hidden,
-                                                                 const float* __restrict__ znorm2,
-                                                                 const int32_t* __restrict__ slot_token,
-                                                                 const int32_t* __restrict__ expert_offset,
-                                                                 const int32_t* __restrict__ expert_count,
-                                                                 const float* __restrict__ row_energy, int d,
-                                                                 CalibState st) {
+__global__ void __launch_bounds__(256) calib_vector_partials_kernel(const __nv_bfloat16* __restrict__ hidden,
+                                                                    const float* __restrict__ znorm2,
+                                                                    const int32_t* __restrict__ slot_token,
+                                                                    const int32_t* __restrict__ expert_offset,
+                                                                    const int32_t* __restrict__ expert_count,
+                                                                    const int32_t* __restrict__ koff,
+                                                                    const float* __restrict__ row_energy, int E, int d,
+                                                                    double* __restrict__ part_z,
+                                                                    double* __restrict__ part_yz,
+                                                                    double* __restrict__ part_s) {
+  __shared__ int s_tok[64];
+  __shared__ float s_inv[64];
+  __shared__ double s_y[64];
+  pdl_launch_dependents();
+  pdl_wait();
+  const int kb = blockIdx.x;
+  if (kb >= koff[E]) return;
+  const int u = expert_of_kblock(koff, E, kb);
+  const int pos0 = (kb - koff[u]) * 64, off = expert_offset[u];
+  const int np = min(64, expert_count[u] - pos0);
+  if (threadIdx.x < 64) {
+    const bool in = int(threadIdx.x) < np;
+    const int t = in ? slot_token[off + pos0 + threadIdx.x] : 0;
+    s_tok[threadIdx.x] = t;
+    s_inv[threadIdx.x] = in ? inv_norm_of(znorm2, t) : 0.f;
+    s_y[threadIdx.x] = in ? log(double(row_energy[off + pos0 + threadIdx.x]) + double(kEnergyEps)) : 0.0;
+  }
+  __syncthreads();
+  const int j = blockIdx.y * 256 + threadIdx.x;
+  if (j < d) {
+    double sz = 0.0, syz = 0.0;
+    for (int p = 0; p < np; ++p) {
+      const double zb = double(bf16_to_f32(hidden[size_t(s_tok[p]) * d + j]) * s_inv[p]);
+      sz += zb;
+      syz += s_y[p] * zb;
+    }
+    part_z[size_t(kb) * d + j] = sz;
+    part_yz[size_t(kb) * d + j] = syz;
+  }
+  if (blockIdx.y == 0 && threadIdx.x == 0) {
+    double sy = 0.0, syy = 0.0, se = 0.0;
+    for (int p = 0; p < np; ++p) {
+      sy += s_y[p];
+      syy += s_y[p] * s_y[p];
+      se += double(row_energy[off + pos0 + p]);
+    }
+    part_s[size_t(kb) * 4 + 0] = sy;
+    part_s[size_t(kb) * 4 + 1] = syy;
+    part_s[size_t(kb) * 4 + 2] = se;
+  }
+}
+
+__global__ void __launch_bounds__(256) calib_vector_reduce_kernel(const int32_t* __restrict__ expert_count,
+                                                                  const int32_t* __restrict__ koff, int d,
+                                                                  const double* __restrict__ part_z,
+                                                                  const double* __restrict__ part_yz,
+                                                                  const double* __restrict__ part_s, CalibState st) {
   pdl_launch_dependents();
   pdl_wait();
   const int u = blockIdx.x, j = blockIdx.y * 256 + threadIdx.x;
-  const int cnt = expert_count[u], off = expert_offset[u];
+  const int cnt = expert_count[u];
   if (cnt == 0) return;
-  double sz = 0.0, syz = 0.0, sy = 0.0, syy = 0.0, se = 0.0;
-  for (int p = 0; p < cnt; ++p) {
-    const int t = slot_token[off + p];
-    const float en = row_energy[off + p];
-    const double y = log(double(en) + double(kEnergyEps));
-    if (j < d) {
-      const double zb = double(bf16_to_f32(hidden[size_t(t) * d + j]) * inv_norm_of(znorm2, t));
-      sz += zb;
-      syz += y * zb;
-    }
-    sy += y;
-    syy += y * y;
-    se += double(en);
-  }
+  const int kb0 = koff[u], kb1 = koff[u + 1];
   if (j < d) {
+    double sz = 0.0, syz = 0.0;
+    for (int kb = kb0; kb < kb1; ++kb) {
+      sz += part_z[size_t(kb) * d + j];
+      syz += part_yz[size_t(kb) * d + j];
+    }
     st.sum_z[size_t(u) * d + j] += sz;
     st.sum_yz[size_t(u) * d + j] += syz;
   }
   if (blockIdx.y == 0 && threadIdx.x == 0) {
+    double sy = 0.0, syy = 0.0, se = 0.0;
+    for (int kb = kb0; kb < kb1; ++kb) {
+      sy += part_s[size_t(kb) * 4 + 0];
+      syy += part_s[size_t(kb) * 4 + 1];
+      se += part_s[size_t(kb) * 4 + 2];
+    }
     st.n[u] += double(cnt);
     st.sum_y[u] += sy;
     st.sum_yy[u] += syy;

@@ -55,6 +55,9 @@ struct CalibScratch {
   __nv_bfloat16* zt_hi;     // [d, ld_cols] transposed normalised inputs, bf16 head
   __nv_bfloat16* zt_lo;     // [d, ld_cols] remainder
   size_t ld_cols;           // padded columns: T*K + 64 per expert, multiple of 64
+  double* part_z;           // [ld_cols/64, d] per-k-block partial sums of the normalised inputs
+  double* part_yz;          // [ld_cols/64, d] ... of y * normalised input
+  double* part_s;           // [ld_cols/64, 4] ... of y, y^2, energy, exp(s-hat)
   size_t bytes;
 };
 
@@ -74,6 +77,9 @@ inline CalibScratch carve_calib_scratch(void* base_ptr, const base_layer_shape& 
   c.koff = static_cast<int32_t*>(take(size_t(s.E + 1) * 4));
   c.zt_hi = static_cast<__nv_bfloat16*>(take(size_t(s.d) * c.ld_cols * 2));
   c.zt_lo = static_cast<__nv_bfloat16*>(take(size_t(s.d) * c.ld_cols * 2));
+  c.part_z = static_cast<double*>(take(c.ld_cols / 64 * size_t(s.d) * 8));
+  c.part_yz = static_cast<double*>(take(c.ld_cols / 64 * size_t(s.d) * 8));
+  c.part_s = static_cast<double*>(take(c.ld_cols / 64 * 4 * 8));
   c.bytes = align_up(off, 1024);
   return c;
 }
@@ -85,8 +91,8 @@ cudaError_t launch_calib_accumulate(const base_layer_shape& s, const Workspace& 
 // Centred ridge solve per expert (conjugate gradients on the fp32 Gram matrix, fp64 vectors).
 cudaError_t launch_calib_solve(const base_layer_shape& s, const CalibState& st, double lambda, cudaStream_t stream);
 // Correction pass: adds sum exp(s-hat) of the routed pairs of this batch (routes must be in the workspace).
-cudaError_t launch_calib_correction(const base_layer_shape& s, const Workspace& ws, const CalibState& st,
-                                    const void* hidden, int T, cudaStream_t stream);
+cudaError_t launch_calib_correction(const base_layer_shape& s, const Workspace& ws, const CalibScratch& sc,
+                                    const CalibState& st, const void* hidden, cudaStream_t stream, int* launches);
 // Intercept correction and rounding to the deployed precision.
 cudaError_t launch_calib_finalize(const base_layer_shape& s, const CalibState& st, void* pred_A_bf16, float* pred_b,
                                   cudaStream_t stream);

@@ -104,39 +104,55 @@ __global__ void __launch_bounds__(kSolveThreads) calib_solve_kernel(CalibState s
   }
 }
 
-// Correction pass: sum over the expert's routed pairs of exp(a_u . zbar_t + b_u), pairs in row order.
-__global__ void __launch_bounds__(256) calib_correction_kernel(const __nv_bfloat16* __restrict__ hidden,
-                                                               const float* __restrict__ znorm2,
-                                                               const int32_t* __restrict__ slot_token,
-                                                               const int32_t* __restrict__ expert_offset,
-                                                               const int32_t* __restrict__ expert_count, int d,
-                                                               CalibState st) {
-  __shared__ double s_val[8];
+// Correction pass: sum over the expert's routed pairs of exp(a_u . zbar_t + b_u), in two levels like
+// the vector statistics: a partial per k-block of 64 pairs (pairs in row order), then the expert's
+// partials in k-block order.
+__global__ void __launch_bounds__(256) calib_correction_partials_kernel(const __nv_bfloat16* __restrict__ hidden,
+                                                                        const float* __restrict__ znorm2,
+                                                                        const int32_t* __restrict__ slot_token,
+                                                                        const int32_t* __restrict__ expert_offset,
+                                                                        const int32_t* __restrict__ expert_count,
+                                                                        const int32_t* __restrict__ koff, int E, int d,
+                                                                        CalibState st, double* __restrict__ part_s) {
+  __shared__ double s_val[64];
   pdl_launch_dependents();
   pdl_wait();
-  const int u = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int cnt = expert_count[u], off = expert_offset[u];
-  if (cnt == 0 || st.n[u] < 1.0) return;
+  const int kb = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (kb >= koff[E]) return;
+  const int u = expert_of_kblock(koff, E, kb);
+  const int pos0 = (kb - koff[u]) * 64, off = expert_offset[u];
+  const int np = min(64, expert_count[u] - pos0);
   const double* a = st.coef_a + size_t(u) * d;
   const double b = st.coef_b[u];
-  double total = 0.0;
-  for (int p0 = 0; p0 < cnt; p0 += 8) {
-    const int p = p0 + warp;
+  for (int p = warp; p < 64; p += 8) {
     double acc = 0.0;
-    if (p < cnt) {
-      const int t = slot_token[off + p];
+    if (p < np) {
+      const int t = slot_token[off + pos0 + p];
       const float inv = inv_norm_of(znorm2, t);
       for (int j = lane; j < d; j += 32) acc += a[j] * double(bf16_to_f32(hidden[size_t(t) * d + j]) * inv);
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) acc += __shfl_down_sync(0xffffffffu, acc, o);
     }
-    if (lane == 0) s_val[warp] = p < cnt ? exp(acc + b) : 0.0;
-    __syncthreads();
-    if (threadIdx.x == 0)
-      for (int w = 0; w < 8; ++w) total += s_val[w];
-    __syncthreads();
+    if (lane == 0) s_val[p] = p < np ? exp(acc + b) : 0.0;
   }
-  if (threadIdx.x == 0) st.sum_p[u] += total;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double total = 0.0;
+    for (int p = 0; p < np; ++p) total += s_val[p];
+    part_s[size_t(kb) * 4 + 3] = total;
+  }
+}
+
+__global__ void __launch_bounds__(32) calib_correction_reduce_kernel(const int32_t* __restrict__ expert_count,
+                                                                     const int32_t* __restrict__ koff,
+                                                                     const double* __restrict__ part_s, CalibState st) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const int u = blockIdx.x;
+  if (threadIdx.x != 0 || expert_count[u] == 0 || st.n[u] < 1.0) return;
+  double total = 0.0;
+  for (int kb = koff[u]; kb < koff[u + 1]; ++kb) total += part_s[size_t(kb) * 4 + 3];
+  st.sum_p[u] += total;
 }
 
 // b_u += log(mean energy / mean exp(s-hat)); coefficients rounded to the deployed precision (bf16
@@ -184,10 +200,16 @@ cudaError_t launch_calib_accumulate(const base_layer_shape& s, const Workspace& 
                  static_cast<const int32_t*>(ws.expert_offset), static_cast<const int32_t*>(ws.expert_count),
                  static_cast<const int32_t*>(sc.koff), s.E, s.d, sc.ld_cols, sc.zt_hi, sc.zt_lo);
   if (e != cudaSuccess) return e;
-  e = launch_pdl(calib_vector_stats_kernel, dim3(s.E, (s.d + 255) / 256), dim3(256), 0, stream, 1, hid,
-                 static_cast<const float*>(ws.znorm2), static_cast<const int32_t*>(ws.slot_token),
+  e = launch_pdl(calib_vector_partials_kernel, dim3(unsigned(sc.ld_cols / 64), (s.d + 255) / 256), dim3(256), 0, stream,
+                 1, hid, static_cast<const float*>(ws.znorm2), static_cast<const int32_t*>(ws.slot_token),
                  static_cast<const int32_t*>(ws.expert_offset), static_cast<const int32_t*>(ws.expert_count),
-                 static_cast<const float*>(sc.row_energy), s.d, st);
+                 static_cast<const int32_t*>(sc.koff), static_cast<const float*>(sc.row_energy), s.E, s.d, sc.part_z,
+                 sc.part_yz, sc.part_s);
+  if (e != cudaSuccess) return e;
+  e = launch_pdl(calib_vector_reduce_kernel, dim3(s.E, (s.d + 255) / 256), dim3(256), 0, stream, 1,
+                 static_cast<const int32_t*>(ws.expert_count), static_cast<const int32_t*>(sc.koff), s.d,
+                 static_cast<const double*>(sc.part_z), static_cast<const double*>(sc.part_yz),
+                 static_cast<const double*>(sc.part_s), st);
   if (e != cudaSuccess) return e;
 
   CUtensorMap m_hi, m_lo;
@@ -206,7 +228,7 @@ cudaError_t launch_calib_accumulate(const base_layer_shape& s, const Workspace& 
   const int grid = std::min(tc_sm_count(), s.E * nb * nb);
   e = launch_pdl(gram_tc_kernel, dim3(grid), dim3(kGramThreads), kGramSmem, stream, 1, m_hi, m_lo, gp);
   if (e != cudaSuccess) return e;
-  *launches += 5;
+  *launches += 6;
   return cudaSuccess;
 }
 
@@ -222,13 +244,23 @@ cudaError_t launch_calib_solve(const base_layer_shape& s, const CalibState& st, 
   return cudaGetLastError();
 }
 
-cudaError_t launch_calib_correction(const base_layer_shape& s, const Workspace& ws, const CalibState& st,
-                                    const void* hidden, int T, cudaStream_t stream) {
-  (void)T;
-  return launch_pdl(calib_correction_kernel, dim3(s.E), dim3(256), 0, stream, 1,
-                    static_cast<const __nv_bfloat16*>(hidden), static_cast<const float*>(ws.znorm2),
-                    static_cast<const int32_t*>(ws.slot_token), static_cast<const int32_t*>(ws.expert_offset),
-                    static_cast<const int32_t*>(ws.expert_count), s.d, st);
+cudaError_t launch_calib_correction(const base_layer_shape& s, const Workspace& ws, const CalibScratch& sc,
+                                    const CalibState& st, const void* hidden, cudaStream_t stream, int* launches) {
+  cudaError_t e = launch_pdl(calib_offsets_kernel, dim3(1), dim3(512), 0, stream, 1,
+                             static_cast<const int32_t*>(ws.expert_count), s.E, sc.koff);
+  if (e != cudaSuccess) return e;
+  e = launch_pdl(calib_correction_partials_kernel, dim3(unsigned(sc.ld_cols / 64)), dim3(256), 0, stream, 1,
+                 static_cast<const __nv_bfloat16*>(hidden), static_cast<const float*>(ws.znorm2),
+                 static_cast<const int32_t*>(ws.slot_token), static_cast<const int32_t*>(ws.expert_offset),
+                 static_cast<const int32_t*>(ws.expert_count), static_cast<const int32_t*>(sc.koff), s.E, s.d, st,
+                 sc.part_s);
+  if (e != cudaSuccess) return e;
+  e = launch_pdl(calib_correction_reduce_kernel, dim3(s.E), dim3(32), 0, stream, 1,
+                 static_cast<const int32_t*>(ws.expert_count), static_cast<const int32_t*>(sc.koff),
+                 static_cast<const double*>(sc.part_s), st);
+  if (e != cudaSuccess) return e;
+  *launches += 3;
+  return cudaSuccess;
 }
 
 cudaError_t launch_calib_finalize(const base_layer_shape& s, const CalibState& st, void* pred_A_bf16, float* pred_b,
