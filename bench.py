@@ -397,6 +397,69 @@ def run_ours(args, cfg, T, M):
         dist.destroy_process_group()
 
 
+def run_calibration(args, cfg, T):
+    """Extra line (not the headline): device calibration of one layer's predictor, App. Calibration Details.
+
+    A step is one statistics batch of T tokens (layer with every original route executed + sufficient
+    statistics); the solve and the correction pass are timed beside it.
+    """
+    import torch
+    from paper_2609_36222_b200 import binding as B, workloads as wl
+    from paper_2609_36222_b200.layer import DeviceLayer, bits_to_device
+    dev = torch.device("cuda:0")
+    torch.cuda.set_device(dev)
+    dl = DeviceLayer(cfg, dev, T_max=T)
+    cal = B.Calibrator(dl.shape, T, dev)
+    n_b = 4
+    hids = [bits_to_device(wl.hidden_bits(cfg, T, 0, 200 + i), dev) for i in range(n_b)]
+
+    def timed(fn, reps):
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(reps):
+            fn(i)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps
+
+    for i in range(max(args.warmup // 4, 3)):
+        cal.accumulate(dl.weights, hids[i % n_b])
+    cal.reset()
+    with ClockSampler(0) as clk:
+        ms_layer = timed(lambda i: B.base_true_removal_costs(dl.shape, dl.weights, hids[i % n_b], dl.workspace), 8)
+        cal.reset()
+        ms_acc = timed(lambda i: cal.accumulate(dl.weights, hids[i % n_b]), n_b * 4)
+        ms_solve = timed(lambda i: cal.solve(1e-2), 1)
+        ms_corr = timed(lambda i: cal.accumulate_correction(dl.weights, hids[i % n_b]), n_b * 4)
+    A, b = cal.finalize()
+    st = cal.statistics()
+    n = st["n"].cpu().numpy()
+    iters = st["cg_iters"].cpu().numpy()
+    active = int((n > 0).sum())
+    gram_bytes = 2.0 * active * cfg.d * cfg.d * 4            # read-modify-write of the touched Gram matrices
+    peaks, kind = measured_peaks()
+    peak = float(peaks.get("hbm_gbs", FALLBACK_HBM_GBS))
+    stat_ms = max(ms_acc - ms_layer, 1e-6)
+    line = {
+        "metric": "calibration_statistics_tokens_per_s", "value": T / ms_acc * 1e3, "unit": "tokens/s", "n_gpus": 1,
+        "steps": n_b * 4, "warmup": max(args.warmup // 4, 3), "ms_per_step": ms_acc, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16 (hi+lo split) x bf16 -> fp32 Gram, fp64 moments",
+        "data": "synthetic",
+        "config": {"workload": f"{cfg.name} layer d={cfg.d} E={cfg.E} K={cfg.K} I={cfg.I}, calibration batches of {T} tokens",
+                   "experts_with_pairs": active, "pairs_per_expert_max": float(n.max())},
+        "parts_ms": {"layer_all_routes_plus_energy": ms_layer, "statistics": stat_ms, "ridge_solve_once": ms_solve,
+                     "correction_batch": ms_corr},
+        "cg_iterations": {"mean": float(iters[n > 0].mean()), "max": int(iters.max())},
+        "roofline": {"bound": "hbm", "kernel": "gram_tc_kernel (with the transposes and vector statistics of the batch)",
+                     "achieved": gram_bytes / (stat_ms * 1e-3) / 1e9, "peak": peak, "unit": "GB/s",
+                     "frac": gram_bytes / (stat_ms * 1e-3) / 1e9 / peak, "traffic": None, "peak_kind": f"of {kind}",
+                     "algorithmic_bytes_per_launch": gram_bytes},
+        "clocks": clk.summary(), "finite": bool(torch.isfinite(A.float()).all() and torch.isfinite(b).all()),
+    }
+    print(json.dumps(line))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -410,13 +473,17 @@ def main():
     ap.add_argument("--no-dense", action="store_true", help="skip the unlimited-budget run")
     ap.add_argument("--profile", action="store_true",
                     help="only the warm-up and the timed steps (for a short run under a profiler)")
+    ap.add_argument("--calib", action="store_true",
+                    help="extra line: device calibration of the predictor on the workload's layer shape")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     from paper_2609_36222_b200 import workloads as wl
     cfg = wl.CONFIGS[args.workload]
     T = args.batch or cfg.T
     M = args.budget
-    if args.impl == "reference":
+    if args.calib:
+        run_calibration(args, cfg, args.batch or 1024)
+    elif args.impl == "reference":
         run_reference(args, cfg, T, M)
     else:
         run_ours(args, cfg, T, M)
