@@ -142,3 +142,44 @@ def test_calibration_error_codes():
     cal = B.Calibrator((cfg.d, cfg.E, cfg.K, cfg.I), 8, DEV)
     with pytest.raises(B.BaseError, match="invalid"):
         cal.solve(0.0)
+
+
+def test_device_fitted_predictor_drives_the_layer():
+    """Calibrate on the device, deploy the coefficients, run the decode layer with them and check it against the
+    oracle given the same coefficients; then the retained energy (Eq. energy_retained) of the selection on held-out
+    tokens: with a predictable energy planted in the experts the fitted score must retain at least as much as the
+    squared-router-weight score (the structure of the paper's selection-rule ablation, not its numbers)."""
+    from gpu_harness import check_layer
+    cfg = wl.CONFIGS["tiny"]
+    sizes = (128, 128, 128, 128, 128, 128)
+    base, batches = _batches(cfg, sizes, planted_alpha=1.0)
+    dl = device_layer_from_host(base, DEV, T_max=128)
+    _, _, _, _, A_dev, b_dev = _run_device(base, batches, dl, with_energies=False)
+    A_bits = wl.f32_to_bf16_bits(A_dev.astype(np.float32)).reshape(cfg.E, cfg.d)   # exact: already bf16 values
+
+    held = HostLayer(cfg, T=64, planted_alpha=1.0)
+    held.hidden_bits = wl.hidden_bits(cfg, 64, 0, 999)
+    held.small["pred_A"] = A_bits
+    held.small["pred_b"] = b_dev.astype(np.float32)
+    dlh = device_layer_from_host(held, DEV)
+    M = 6
+    rep = check_layer(held, dlh, M)                       # parity of the layer under the deployed predictor
+
+    hid = bits_to_device(held.hidden_bits, DEV)
+    lg = torch.from_numpy(O.router_logits(held.z, held.router_w, held.router_bias)).to(DEV)
+    tc, _, _, _ = B.base_true_removal_costs(dlh.shape, dlh.weights, hid, dlh.workspace, router_logits=lg)
+    d_star, _, _ = B.base_aggregate_select(tc, M)
+
+    def retained(score_rule):
+        out = torch.empty(64, cfg.d, dtype=torch.float32, device=DEV)
+        dbg, dt = B.alloc_debug(64, cfg.E, cfg.K, M, DEV)
+        B.base_moe_decode_layer(dlh.shape, dlh.weights, hid, M, out, dlh.workspace, router_logits=lg, debug=dbg,
+                                score_rule=score_rule)
+        return float(B.base_energy_retained(d_star, dt["active_mask"], M).cpu()[0])
+
+    er_fit, er_w2 = retained(B.SCORE_PREDICTED), retained(B.SCORE_WEIGHT_SQ)
+    ref_er = O.energy_retained(rep["ref"]["mask"], d_star.cpu().numpy().astype(np.float64), M)
+    assert abs(er_fit - ref_er) <= 1e-5 or rep["forced"]
+    assert 0.0 < er_w2 <= 1.0 + 1e-6 and er_fit <= 1.0 + 1e-6
+    assert er_fit >= er_w2 - 1e-3, (er_fit, er_w2)
+    assert er_fit > 0.9
