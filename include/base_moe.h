@@ -60,6 +60,9 @@ enum { BASE_SCORE_PREDICTED = 0,   /* Eq. log_energy_predictor: sum of w^2 exp(a
        BASE_SCORE_TOP1_UNION = 4 };/* number of tokens whose first choice the expert is (positive on the top-1 union) */
 enum { BASE_FILL_BACKFILL = 0,     /* Sec. 3.5: next-preferred experts inside the active set */
        BASE_FILL_DROP = 1 };       /* fill-rule ablation: unavailable routes are removed */
+enum { BASE_ROUTER_NORM_TOPK = 0,  /* w = softmax score renormalised over the token's top-K (sums to 1) */
+       BASE_ROUTER_NORM_ALL = 1 }; /* w = plain softmax probability over all experts (the convention of the paper's
+                                      other two models, Sec. 4.1); the top-K weights then sum to less than 1 */
 
 /*
  * Predicted removal costs of the routed pairs (Eq. log_energy_predictor; scoring kernel of
@@ -128,6 +131,7 @@ typedef struct {
   int out_is_fp32;          /* 0: out is bf16 [T,d]; 1: out is fp32 [T,d] */
   int ffn_impl;             /* 0: default (tensor-core streaming kernels); 1: simple CUDA-core kernels */
   int score_rule;           /* BASE_SCORE_*: what a routed pair contributes to its expert's batch score */
+  int router_norm;          /* BASE_ROUTER_NORM_*: denominator of the router weights w (and of the paper-rule gates) */
 } base_layer_options;
 
 /* Bytes of device workspace base_moe_decode_layer needs for up to T_max tokens (0 on bad shape). */

@@ -27,6 +27,8 @@ GATE_RULE_PAPER = 0       # Sec. 3.5: denominator from the token's ORIGINAL top-
 GATE_RULE_RENORM = 1      # OEA-style: renormalise over the executed experts
 FILL_BACKFILL = 0         # Sec. 3.5: next-preferred experts inside the active set
 FILL_DROP = 1             # fill-rule ablation: unavailable routes are simply removed
+ROUTER_NORM_TOPK = 0      # router weights renormalised over the token's top-K
+ROUTER_NORM_ALL = 1       # plain softmax over all experts, no renormalisation after the top-K
 # what a routed pair contributes to its expert's batch score (App. Selection-Rule Ablation)
 SCORE_PREDICTED = 0       # w^2 exp(a . z-bar + b): the method (Eq. log_energy_predictor)
 SCORE_WEIGHT_SQ = 1       # squared router-weight sum
@@ -50,18 +52,26 @@ def rank_desc(values):
     return np.argsort(-v, kind="stable")
 
 
-def route_topk(logits, K):
-    """Token-choice top-K routing (Sec. 3.1) with softmax scores renormalised over R_t.
+def route_topk(logits, K, router_norm=ROUTER_NORM_TOPK):
+    """Token-choice top-K routing (Sec. 3.1).
+
+    ROUTER_NORM_TOPK: softmax scores renormalised over R_t (sum_u w_{t,u} = 1), the reading used for the
+    Qwen3 and Mixtral shapes. ROUTER_NORM_ALL: plain softmax probabilities over all experts, not
+    renormalised after the top-K (the convention of the paper's other two models, Sec. 4.1); then
+    sum_u w_{t,u} < 1. Only the denominator S changes.
 
     Returns order [T,E] (full ranking by logit), R [T,K], q [T,E] = exp(l - max_e l),
-    S [T] = sum_{u in R_t} q, w [T,K] = q[R_t] / S_t  (so sum_u w_{t,u} = 1).
+    S [T] = the denominator, w [T,K] = q[R_t] / S_t.
     """
     l = np.asarray(logits, np.float64)
     T, E = l.shape
     order = np.stack([rank_desc(l[t]) for t in range(T)])
     R = order[:, :K]
     q = np.exp(l - l.max(axis=1, keepdims=True))
-    S = np.take_along_axis(q, R, axis=1).sum(axis=1)
+    if router_norm == ROUTER_NORM_ALL:
+        S = q.sum(axis=1)
+    else:
+        S = np.take_along_axis(q, R, axis=1).sum(axis=1)
     w = np.take_along_axis(q, R, axis=1) / S[:, None]
     return order, R, q, S, w
 
@@ -175,14 +185,15 @@ def execute(z, ids, gates, expert_weights):
 # ----------------------------------------------------------------------------- the layer
 
 def moe_decode_layer(z, logits, pred_A, pred_b, expert_weights, K, M,
-                     gate_rule=GATE_RULE_PAPER, fill=FILL_BACKFILL, forced_mask=None, score_rule=SCORE_PREDICTED):
+                     gate_rule=GATE_RULE_PAPER, fill=FILL_BACKFILL, forced_mask=None, score_rule=SCORE_PREDICTED,
+                     router_norm=ROUTER_NORM_TOPK):
     """One BASE decode step of one MoE layer, in the paper's order:
     route -> predict costs -> aggregate -> top-M -> restrict routes -> execute.
 
     ``forced_mask`` replaces the predicted selection (used to compare near-ties).
     Returns a dict with every intermediate.
     """
-    order, R, q, S, w = route_topk(logits, K)
+    order, R, q, S, w = route_topk(logits, K, router_norm)
     costs = predict_costs(z, R, w, pred_A, pred_b, score_rule)
     scores = aggregate(costs)
     sel, mask = select_top(scores, M)

@@ -84,6 +84,7 @@ int enqueue_routing(const LayerCall& c, const Workspace& ws, cudaStream_t st, in
   ra.gate_rule = c.opt.gate_rule;
   ra.fill_rule = c.opt.fill_rule;
   ra.score_rule = c.opt.score_rule;
+  ra.router_norm = c.opt.router_norm;
   ra.ws = ws;
   ra.dbg = c.dbg;
   e = launch_routing(ra, st);
@@ -139,6 +140,7 @@ int check_layer_args(const base_layer_shape* shape, const base_layer_weights* w,
     if (opt->fill_rule != BASE_FILL_BACKFILL && opt->fill_rule != BASE_FILL_DROP) return BASE_ERR_INVALID_ARG;
     if (opt->ffn_impl != 0 && opt->ffn_impl != 1) return BASE_ERR_INVALID_ARG;
     if (opt->score_rule < BASE_SCORE_PREDICTED || opt->score_rule > BASE_SCORE_TOP1_UNION) return BASE_ERR_INVALID_ARG;
+    if (opt->router_norm != BASE_ROUTER_NORM_TOPK && opt->router_norm != BASE_ROUTER_NORM_ALL) return BASE_ERR_INVALID_ARG;
   }
   return BASE_OK;
 }

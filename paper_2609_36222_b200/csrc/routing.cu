@@ -404,10 +404,19 @@ __global__ void __launch_bounds__(kRoutingThreads) routing_kernel(RoutingArgs a)
     }
     const uint32_t taken = avail0 & ~avail;
     float q[NV], qs = 0.f;
+    if (a.router_norm == BASE_ROUTER_NORM_TOPK) {   // the denominator is the sum over the token's top-K
 #pragma unroll
-    for (int i = 0; i < NV; ++i) {
-      q[i] = ((taken >> i) & 1u) ? expf(l[i] - m) : 0.f;
-      qs += q[i];
+      for (int i = 0; i < NV; ++i) {
+        q[i] = ((taken >> i) & 1u) ? expf(l[i] - m) : 0.f;
+        qs += q[i];
+      }
+    } else {                                        // ... or over all experts (plain softmax)
+#pragma unroll
+      for (int i = 0; i < NV; ++i) {
+        const float qa = ((avail0 >> i) & 1u) ? expf(l[i] - m) : 0.f;
+        q[i] = ((taken >> i) & 1u) ? qa : 0.f;
+        qs += qa;
+      }
     }
     const float S_t = warp_sum(qs);
     // what a routed pair adds to its expert's score: the method's predicted removal cost (the loop the

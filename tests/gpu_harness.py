@@ -50,15 +50,16 @@ def run_gpu(dl, hidden_dev, M, logits=None, forced_mask=None, out_dtype=torch.fl
 
 
 def check_layer(host, dl, M, gate_rule=0, fill_rule=0, out_dtype=torch.float32, ffn_impl=0, check_out=True,
-                score_rule=0):
+                score_rule=0, router_norm=0):
     """Run oracle and CUDA path on the same inputs and compare every intermediate. Returns a report."""
     cfg = host.cfg
     z = host.z
     logits = O.router_logits(z, host.router_w, host.router_bias)
     ref = O.moe_decode_layer(z, logits, host.pred_A, host.pred_b, host.expert_weights, cfg.K, M,
-                             gate_rule=gate_rule, fill=fill_rule, score_rule=score_rule)
+                             gate_rule=gate_rule, fill=fill_rule, score_rule=score_rule, router_norm=router_norm)
     hidden_dev = bits_to_device(host.hidden_bits, dl.device)
-    kw = dict(gate_rule=gate_rule, fill_rule=fill_rule, ffn_impl=ffn_impl, out_dtype=out_dtype, score_rule=score_rule)
+    kw = dict(gate_rule=gate_rule, fill_rule=fill_rule, ffn_impl=ffn_impl, out_dtype=out_dtype, score_rule=score_rule,
+              router_norm=router_norm)
     got = run_gpu(dl, hidden_dev, M, logits=logits, **kw)
 
     assert got["status"][0] == 0

@@ -115,6 +115,10 @@ def test_other_model_shapes(E, K, T):
     for M in cfg.budgets + (E,):
         check_layer(host, dl, M)
     check_layer(host, dl, 20, gate_rule=B.GATE_RENORM, fill_rule=B.FILL_DROP)
+    # those two models do not renormalise the router weights over the top-K
+    rep = check_layer(host, dl, 20, router_norm=B.ROUTER_NORM_ALL)
+    assert (rep["ref"]["w"].sum(axis=1) < 1.0).all()
+    check_layer(host, dl, 8, router_norm=B.ROUTER_NORM_ALL, gate_rule=B.GATE_RENORM)
 
 
 # ------------------------------------------------------------------------------- edge cases

@@ -299,6 +299,11 @@ def test_primitives_against_torch():
     np.testing.assert_array_equal(R, ti.numpy())
     np.testing.assert_allclose(w, (tv / tv.sum(dim=1, keepdim=True)).numpy(), rtol=1e-12)
     np.testing.assert_array_equal(order, torch.argsort(torch.from_numpy(logits), dim=1, descending=True, stable=True).numpy())
+    # router weights without renormalisation over the top-K: the softmax probabilities themselves
+    _, R2, _, S2, w2 = O.route_topk(logits, 3, O.ROUTER_NORM_ALL)
+    np.testing.assert_array_equal(R2, ti.numpy())
+    np.testing.assert_allclose(w2, tv.numpy(), rtol=1e-12)
+    assert (w2.sum(axis=1) < 1).all() and (S2 > S).all()
     zz = r.standard_normal((4, 12))
     np.testing.assert_allclose(O.normalise(zz), F.normalize(torch.from_numpy(zz), dim=1).numpy(), rtol=1e-14)
     np.testing.assert_allclose(O.router_logits(x, Wg, np.arange(7.0)),
