@@ -211,7 +211,14 @@ def run_ours(args, cfg, T, M):
     ws = B.alloc_workspace(max(B.layer_workspace_bytes(*shape, T), B.stack_workspace_bytes(*shape, T)), dev)
     layer_ids = multi.replica_layer_ids(rank, n_rep)
     base_layer = layer_ids[0]
-    layers = [DeviceLayer(cfg, dev, layer=l, T_max=T, workspace=ws) for l in layer_ids]
+    def small_of(l):
+        if args.bias_scale == 1.0:
+            return None
+        sm = wl.small_tensors(cfg, 0, l)
+        sm["router_bias"] = wl.router_bias(cfg, 0, l, args.bias_scale)   # sensitivity row: flatter routing
+        return sm
+
+    layers = [DeviceLayer(cfg, dev, layer=l, T_max=T, workspace=ws, small=small_of(l)) for l in layer_ids]
     hidden = [bits_to_device(wl.hidden_bits(cfg, T, layer=l), dev) for l in layer_ids]
     out = torch.empty(T, cfg.d, dtype=torch.bfloat16, device=dev)
     nd_buf = torch.zeros(max(n_rep, 1), dtype=torch.int32, device=dev)
@@ -359,7 +366,8 @@ def run_ours(args, cfg, T, M):
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {
             "workload": f"{cfg.name} {'stack L=%d ' % cfg.layers if stack else 'layer '}d={cfg.d} E={cfg.E} K={cfg.K} "
-                        f"I={cfg.I} batch={T} budget={M}",
+                        f"I={cfg.I} batch={T} budget={M}"
+                        + ("" if args.bias_scale == 1.0 else f" [sensitivity row: router bias x {args.bias_scale:g}]"),
             "l2": f"cold: {n_rep} independently seeded weight replicas rotated between steps "
                   f"({mean_nd * cfg.expert_bytes / 1e6:.0f} MB dispatched per step vs 126 MB L2)",
             "n_dispatched_mean": mean_nd, "replicas": n_rep, "timing": "CUDA events around graph replays",
@@ -473,6 +481,9 @@ def main():
     ap.add_argument("--no-dense", action="store_true", help="skip the unlimited-budget run")
     ap.add_argument("--profile", action="store_true",
                     help="only the warm-up and the timed steps (for a short run under a profiler)")
+    ap.add_argument("--bias-scale", type=float, default=1.0,
+                    help="scale of the Zipf router bias (1 = the workload as defined; 0 = flat routing, a sensitivity "
+                         "row that is not one of the defined configurations)")
     ap.add_argument("--calib", action="store_true",
                     help="extra line: device calibration of the predictor on the workload's layer shape")
     args = ap.parse_args()
