@@ -85,6 +85,7 @@ int enqueue_routing(const LayerCall& c, const Workspace& ws, cudaStream_t st, in
   ra.fill_rule = c.opt.fill_rule;
   ra.score_rule = c.opt.score_rule;
   ra.router_norm = c.opt.router_norm;
+  ra.ffn_first_ticket = c.opt.ffn_impl == 1 ? 0 : ffn_tc_static_units(s, c.T, c.budget, ws);
   ra.ws = ws;
   ra.dbg = c.dbg;
   e = launch_routing(ra, st);

@@ -112,7 +112,7 @@ struct FfnParams {
   const int32_t* slot_token;     // [rows] token of every sorted row
   const int32_t* exec_ids;       // [T,K] executed experts per token (-1: none)
   const int32_t* token_slot;     // [T,K] sorted row of every executed route
-  int T, K;
+  int T, K, E;
   int I, d;
   int tiles1, tiles2;   // work units per segment: I/64 gate/up tiles, d/128 down tiles
   int steps1, steps2;   // pipeline stages per unit: ceil(d/64 / 2), ceil(kb2 / 2)
@@ -260,21 +260,49 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
         n_units = u1 + n_seg * down_units_per_seg;
         final_known = true;
       };
+      // The first unit of a dense batch is static: CTA c takes gate/up unit c (the ticket counter starts
+      // behind these), and it needs nothing but the expert id, so the producer polls that one entry of
+      // the early list and issues its first weight box a single L2 round trip after the routing kernel
+      // has written it. (An entry is -1 until then; a unit past the early list waits for the final one.)
+      int u_cur;
+      Unit un_next{};
+      int early_units = -1;
       if (kDense) {
-        int flag = 0;
-        const long long t0 = clock64();
+        u_cur = blockIdx.x;
+        const int j = u_cur / p.tiles1;
+        int e0 = -1;
+        if (j < p.E) {
+          const long long t0 = clock64();
 #pragma unroll 1
-        for (uint32_t it = 0; it < kSpinLimit; ++it) {
-          flag = ld_acquire(p.counters + kCtrEarly);
-          if (flag > 0) break;
-          __nanosleep(128);
-          if ((it & 63u) == 63u && clock64() - t0 > kEarlyPollCycles) break;
+          for (uint32_t it = 0; it < kSpinLimit; ++it) {
+            e0 = ld_acquire(p.gu_expert + j);
+            if (e0 >= 0) break;
+            const int flag = ld_acquire(p.counters + kCtrEarly);
+            if (flag > 0 && u_cur >= (flag - 1) * p.tiles1) break;   // the early list ends before this unit
+            __nanosleep(128);
+            if ((it & 63u) == 63u && clock64() - t0 > kEarlyPollCycles) break;
+          }
         }
-        if (flag > 0) u1 = n_units = (flag - 1) * p.tiles1;   // else: no early list seen, wait for the final one
+        if (e0 >= 0) {
+          un_next.phase = 1;
+          un_next.seg = j;
+          un_next.expert = e0;
+          un_next.tile = u_cur - j * p.tiles1;
+          un_next.kb0 = 0;
+          un_next.offset = 0;
+          un_next.count = p.T;
+          un_next.npad = (p.T + 15) & ~15;
+          u1 = n_units = u_cur + 1;   // provisional: the length of the early list is read with the next ticket
+        } else {
+          make_final();
+          early_units = 0;
+          un_next = decode_unit<kSplit, kDense>(p, min(u_cur, max(n_units - 1, 0)), u1);
+        }
+      } else {
+        u_cur = atomicAdd(p.counters + kCtrTicket, 1);
+        make_final();
+        un_next = decode_unit<kSplit, kDense>(p, min(u_cur, max(n_units - 1, 0)), u1);
       }
-      int u_cur = atomicAdd(p.counters + kCtrTicket, 1);
-      if (!kDense || u_cur >= n_units) make_final();
-      Unit un_next = decode_unit<kSplit, kDense>(p, min(u_cur, max(n_units - 1, 0)), u1);
       while (ok && u_cur < n_units) {
         const Unit un = un_next;
         int u_next = 0x7fffffff;
@@ -356,6 +384,20 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
             phase ^= 1u;
           }
           if (st == 0) {
+            if (kDense && !final_known && early_units < 0) {
+              // length of the early list: published right after the entries this CTA has already seen
+              int flag = 0;
+              const long long t0 = clock64();
+#pragma unroll 1
+              for (uint32_t it = 0; it < kSpinLimit; ++it) {
+                flag = ld_acquire(p.counters + kCtrEarly);
+                if (flag > 0) break;
+                __nanosleep(64);
+                if ((it & 63u) == 63u && clock64() - t0 > kEarlyPollCycles) break;
+              }
+              early_units = flag > 0 ? (flag - 1) * p.tiles1 : 0;
+              u1 = n_units = max(early_units, u_cur + 1);
+            }
             if (kDense && !final_known && u_next >= n_units) make_final();   // past the early list
             if (u_next < n_units) un_next = decode_unit<kSplit, kDense>(p, u_next, u1);
           }
@@ -774,7 +816,24 @@ cudaError_t launch_kernel(const MapSet& m1, const MapSet& m2, const FfnParams& p
                       : launch_variant<kMaxN, 1, kDense>(m1, m2, p, max_units, st);
 }
 
+// K split of the down pass (see launch_ffn_tc) and the launch grid, shared with the routing set-up.
+int choose_split(const base_layer_shape& s, int T, int budget, int ypair_copies) {
+  const int kb_all = s.I / kBlockK;
+  const int expect_experts = std::min(std::min(budget, s.E), T * s.K);
+  const int down_units = (s.d / 128) * expect_experts;
+  int want = down_units >= 2 * sm_count() ? 1 : kMaxSplit;
+  while (want > 1 && (kb_all < 8 * want || want > ypair_copies)) want >>= 1;
+  return want;
+}
+
 }  // namespace
+
+int ffn_tc_static_units(const base_layer_shape& s, int T, int budget, const Workspace& ws) {
+  if (T > 128) return 0;   // batches that gather their tokens take every unit from the ticket counter
+  const int segs = max_segments(s.E, T, s.K);
+  const int max_units = segs * (s.I / 64 + (s.d / 128) * choose_split(s, T, budget, ws.ypair_copies));
+  return std::min(sm_count(), max_units);
+}
 
 bool tc_map_rows_kblocks(const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows, uint32_t box_kb,
                           CUtensorMap* out) {
@@ -823,6 +882,7 @@ cudaError_t launch_ffn_tc(const base_layer_shape& s, const base_layer_weights& w
   p.token_slot = ws.token_slot;
   p.T = T;
   p.K = s.K;
+  p.E = s.E;
   p.I = s.I;
   p.d = s.d;
 #ifdef BASE_FFN_CYCLES
@@ -836,11 +896,7 @@ cudaError_t launch_ffn_tc(const base_layer_shape& s, const base_layer_weights& w
   // of at least 8 k-blocks, as many as the workspace holds partial-sum copies for. (On Mixtral-sized
   // experts two chunks and four measured within 2% of each other; more copies cost the combine more.)
   const int kb_all = s.I / kBlockK;
-  const int expect_experts = std::min(std::min(budget, s.E), T * s.K);
-  const int down_units = p.tiles2 * expect_experts;
-  int want = down_units >= 2 * sm_count() ? 1 : kMaxSplit;
-  while (want > 1 && (kb_all < 8 * want || want > ws.ypair_copies)) want >>= 1;
-  p.ksplit = want;
+  p.ksplit = choose_split(s, T, budget, ws.ypair_copies);
   p.ypair_stride = ws.ypair_stride;
   p.kb2 = p.ksplit == 1 ? kb_all
                         : ((kb_all + p.ksplit - 1) / p.ksplit + int(kKbPerStage) - 1) / int(kKbPerStage) * int(kKbPerStage);

@@ -10,6 +10,8 @@ namespace base {
 bool tc_map_rows_kblocks(const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows, uint32_t box_kb,
                           CUtensorMap* out);
 int tc_sm_count();
+// Gate/up units that the FFN kernel's CTAs take statically (CTA c takes unit c); the ticket counter starts behind them.
+int ffn_tc_static_units(const base_layer_shape& s, int T, int budget, const Workspace& ws);
 cudaError_t launch_ffn_tc(const base_layer_shape& s, const base_layer_weights& w, const void* hidden,
                           const Workspace& ws, int T, int budget, cudaStream_t st, int* launches, int* n_split);
 }

@@ -355,8 +355,9 @@ __global__ void __launch_bounds__(kRoutingThreads) routing_kernel(RoutingArgs a)
   // cannot start before every CTA of this kernel has passed launch_dependents.
   if (cta == 0) {
     for (int i = threadIdx.x; i < a.max_segs * kMaxSplit; i += kRoutingThreads) a.ws.counters[kCtrReady + i] = 0;
+    for (int e = threadIdx.x; e < E; e += kRoutingThreads) a.ws.gu_expert[e] = -1;   // "not yet known"
     if (threadIdx.x == 0) {
-      a.ws.counters[kCtrTicket] = 0;
+      a.ws.counters[kCtrTicket] = a.ffn_first_ticket;
       a.ws.counters[kCtrGather] = 0;
       a.ws.counters[kCtrEarly] = 0;
       a.ws.counters[kCtrGuUnits] = 0;
