@@ -353,7 +353,9 @@ __global__ void __launch_bounds__(kRoutingThreads) routing_kernel(RoutingArgs a)
   // running, so its scheduling counters are cleared here, before it is allowed to launch: the
   // previous FFN kernel has completed (completion is transitive through the waits), and the next one
   // cannot start before every CTA of this kernel has passed launch_dependents.
-  if (cta == 0) {
+  // (Done by the last CTA of the cluster, which has the fewest tokens to route, so that the device
+  // fence below stays off the path to the selection.)
+  if (cta == kClusterCtas - 1) {
     for (int i = threadIdx.x; i < a.max_segs * kMaxSplit; i += kRoutingThreads) a.ws.counters[kCtrReady + i] = 0;
     for (int e = threadIdx.x; e < E; e += kRoutingThreads) a.ws.gu_expert[e] = -1;   // "not yet known"
     if (threadIdx.x == 0) {
