@@ -340,6 +340,7 @@ __global__ void __launch_bounds__(kRoutingThreads) routing_kernel(RoutingArgs a)
   __shared__ int32_t s_wsum[kRoutingWarps], s_wseg[kRoutingWarps], s_wlate[kRoutingWarps];
   __shared__ int s_status, s_n_early;
   __shared__ uint8_t s_early[kMaxE];
+  __shared__ int16_t s_rank[kMaxE];
 
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int cta = int(cluster_cta_rank());
@@ -515,15 +516,9 @@ __global__ void __launch_bounds__(kRoutingThreads) routing_kernel(RoutingArgs a)
     if (e < E && part == 0) {
       const uint8_t in = r < M;
       s_mask[e] = a.forced_mask ? (a.forced_mask[e] != 0) : in;
-      if (cta == 0) {
-        a.ws.mask[e] = in;
-        if (in) a.ws.selected[r] = e;
-        if (a.dbg.active_mask) a.dbg.active_mask[e] = in;
-        if (in && a.dbg.selected_ids) a.dbg.selected_ids[r] = e;
-      }
+      s_rank[e] = int16_t(r);
     }
   }
-  for (int i = threadIdx.x; i < ((T + 31) >> 5) * E; i += kRoutingThreads) s_bal[i] = 0u;
   __syncthreads();
   // Early expert list for the FFN kernel, published as soon as the selection stands: every score rule
   // sums over routed pairs only, so a selected expert with a positive score has an original route,
@@ -551,7 +546,17 @@ __global__ void __launch_bounds__(kRoutingThreads) routing_kernel(RoutingArgs a)
     __syncthreads();   // orders every thread's list entries before the release below (cumulative)
     if (threadIdx.x == 0)
       asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(a.ws.counters + kCtrEarly), "r"(total + 1) : "memory");
+    // what the FFN kernel does not wait for comes after the list
+    for (int e = threadIdx.x; e < E; e += kRoutingThreads) {
+      const int r = s_rank[e];
+      const uint8_t in = r < M;
+      a.ws.mask[e] = in;
+      if (in) a.ws.selected[r] = e;
+      if (a.dbg.active_mask) a.dbg.active_mask[e] = in;
+      if (in && a.dbg.selected_ids) a.dbg.selected_ids[r] = e;
+    }
   }
+  for (int i = threadIdx.x; i < ((T + 31) >> 5) * E; i += kRoutingThreads) s_bal[i] = 0u;
   RT_STAMP(4)
 
   // ---- ... and the restricted routes of this CTA's tokens. Original routes that are still active
