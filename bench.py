@@ -248,26 +248,45 @@ def run_ours(args, cfg, T, M):
     mean_nd = float(nd.mean())
 
     def capture(budget):
+        # single-step graphs (one per weight replica) and, for single layers, one graph that holds a step
+        # on every replica back to back -- the way consecutive layers of a model sit in one graph, so that
+        # programmatic dependent launch also overlaps one step's set-up with the previous step's tail
         graphs = []
         for r in range(1 if stack else n_rep):
             g = torch.cuda.CUDAGraph()
             with torch.cuda.graph(g, stream=stream):
                 step_eager(r, budget)
             graphs.append(g)
-        return graphs
+        chain = None
+        if not stack and n_rep > 1 and not args.single_step_graphs:
+            chain = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(chain, stream=stream):
+                for r in range(n_rep):
+                    step_eager(r, budget)
+        return graphs, chain
 
-    def timed(graphs, steps, warmup):
+    def timed(captured, steps, warmup):
+        graphs, chain = captured
+
+        def run(n):            # exactly n steps: chains of len(graphs) steps, then single steps
+            done = 0
+            if chain is not None:
+                while done + len(graphs) <= n:
+                    chain.replay()
+                    done += len(graphs)
+            while done < n:
+                graphs[done % len(graphs)].replay()
+                done += 1
+
         with torch.cuda.stream(stream):
-            for i in range(warmup):
-                graphs[i % len(graphs)].replay()
+            run(warmup)
             stream.synchronize()
             if dist is not None:
                 dist.barrier()
             torch.cuda.synchronize()
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record(stream)
-            for i in range(steps):
-                graphs[(warmup + i) % len(graphs)].replay()
+            run(steps)
             e1.record(stream)
             e1.synchronize()
             torch.cuda.synchronize()
@@ -370,7 +389,8 @@ def run_ours(args, cfg, T, M):
                         + ("" if args.bias_scale == 1.0 else f" [sensitivity row: router bias x {args.bias_scale:g}]"),
             "l2": f"cold: {n_rep} independently seeded weight replicas rotated between steps "
                   f"({mean_nd * cfg.expert_bytes / 1e6:.0f} MB dispatched per step vs 126 MB L2)",
-            "n_dispatched_mean": mean_nd, "replicas": n_rep, "timing": "CUDA events around graph replays",
+            "n_dispatched_mean": mean_nd, "replicas": n_rep, "timing": ("CUDA events around graph replays, one graph per step" if (stack or n_rep == 1 or args.single_step_graphs)
+                       else f"CUDA events around graph replays, {n_rep} consecutive steps (one per replica) per graph"),
             "multi_gpu": "independent replicas per rank, no collective" if world > 1 else "single GPU",
         },
         "hbm": {"algorithmic_bytes_per_step": step_bytes, "gbs": gbs, "frac_of_nominal_8tbs": gbs / NOMINAL_HBM_GBS,
@@ -481,6 +501,8 @@ def main():
     ap.add_argument("--no-dense", action="store_true", help="skip the unlimited-budget run")
     ap.add_argument("--profile", action="store_true",
                     help="only the warm-up and the timed steps (for a short run under a profiler)")
+    ap.add_argument("--single-step-graphs", action="store_true",
+                    help="replay one graph per step instead of one graph per round of weight replicas")
     ap.add_argument("--bias-scale", type=float, default=1.0,
                     help="scale of the Zipf router bias (1 = the workload as defined; 0 = flat routing, a sensitivity "
                          "row that is not one of the defined configurations)")
