@@ -102,7 +102,7 @@ __device__ __forceinline__ void aggregate_columns(const float* __restrict__ cost
     const int g = idx / E_pad, e = idx - g * E_pad;
     float acc = 0.f;
     if (e < E) {
-#pragma unroll 8
+#pragma unroll 16   // a batch of 64 tokens and 128 experts has all its loads in flight at once; the order of the sum is fixed
       for (int t = g; t < T; t += G) acc += costs[size_t(t) * E + e];
     }
     s_part[idx] = acc;
