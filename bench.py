@@ -204,7 +204,7 @@ def run_ours(args, cfg, T, M):
     if stack:
         n_rep = cfg.layers
     else:
-        n_rep = max(2, min(8, int(np.ceil(4 * 126e6 / max(1, min(M, cfg.E) * cfg.expert_bytes))) + 1))
+        n_rep = max(4, min(8, int(np.ceil(4 * 126e6 / max(1, min(M, cfg.E) * cfg.expert_bytes))) + 1))
         if cfg.E * cfg.expert_bytes * n_rep > 40e9:
             n_rep = max(2, int(40e9 // (cfg.E * cfg.expert_bytes)))
     shape = (cfg.d, cfg.E, cfg.K, cfg.I)
