@@ -136,9 +136,10 @@ def test_ragged_batch_sizes(T):
 
 @pytest.mark.parametrize("d,E,K,I,T,M", [(256, 32, 8, 128, 1024, 12),      # T and T*K at the compiled limits
                                             (256, 512, 16, 64, 512, 40),      # E, K and T*K at the compiled limits
-                                            (256, 512, 16, 64, 3, 512)])      # the same expert count, a tiny batch
+                                            (256, 512, 16, 64, 3, 512),       # the same expert count, a tiny batch
+                                            (8192, 4, 2, 64, 16, 3)])         # the widest model dimension
 def test_maximum_sizes(d, E, K, I, T, M):
-    """Shapes at the limits the library is compiled for (1024 tokens, 8192 routed pairs, 512 experts, top-16);
+    """Shapes at the limits the library is compiled for (1024 tokens, 8192 routed pairs, 512 experts, top-16, d = 8192);
     d and I are kept small so that the oracle finishes in seconds."""
     cfg = wl.LayerConfig(f"max_E{E}_K{K}_T{T}", d=d, E=E, K=K, I=I, T=T, budgets=(M,))
     host = HostLayer(cfg, T=T)
