@@ -307,7 +307,7 @@ def run_ours(args, cfg, T, M):
     # Six events per replica are recorded by the library between the kernels of the step; the step is captured
     # in a graph with those records as nodes, so the replay has no host launch gaps.
     n_prof = min(args.steps, 60)
-    ffn_us, stage_us = None, None
+    ffn_us, stage_us, event_pair_us = None, None, None
     if not args.profile:
         n_g = 1 if stack else n_rep
         evs = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(n_g)]
@@ -334,7 +334,9 @@ def run_ours(args, cfg, T, M):
                         samples[name].append(evs[r][j].elapsed_time(evs[r][j + 1]) * 1e3)
         # (in a stack every layer re-records the events, so these are the last layer's kernels)
         stage_us = {name: statistics.mean(v) for name, v in samples.items()}
-        stage_us.pop("gather", None)   # only the cross-check FFN has a gather kernel; here the interval is two event records
+        # only the cross-check FFN has a gather kernel: on this path that interval holds nothing but its two event
+        # records, i.e. it measures what an event pair adds to every other interval
+        event_pair_us = stage_us.pop("gather", None)
         ffn_us = stage_us["expert_ffn"]
 
     # ---- unlimited budget (dense batch-union step) for the speed-up, same protocol
@@ -411,6 +413,10 @@ def run_ours(args, cfg, T, M):
                             "traffic": NCU_FFN_TRAFFIC.get((cfg.name, T, M)),
                             "us_per_launch": ffn_us, "peak_kind": f"of {peak_kind}",
                             "algorithmic_bytes_per_launch": fb}
+        if event_pair_us is not None and 0 < event_pair_us < ffn_us:
+            # context only: `frac` above keeps the raw event figure; the ncu launch list in profiles/ agrees with this one
+            line["roofline"]["event_pair_overhead_us"] = event_pair_us
+            line["roofline"]["frac_less_event_overhead"] = fb / ((ffn_us - event_pair_us) * 1e-6) / 1e9 / hbm_peak
         line["kernel_us"] = stage_us
     # CPU baseline: the oracle, as it stands, on this machine's host cores
     if not args.no_cpu and not args.profile:
