@@ -406,60 +406,46 @@ __global__ void __launch_bounds__(kRoutingThreads) routing_kernel(RoutingArgs a)
         myid = gi;
       }
     }
-    const uint32_t taken = avail0 & ~avail;
-    float q[NV], qs = 0.f;
-    if (a.router_norm == BASE_ROUTER_NORM_TOPK) {   // the denominator is the sum over the token's top-K
+    // From here on lane k works for the k-th route only (one exponential and one division per lane
+    // instead of one per entry): its softmax score, the denominator, its weight and what the pair
+    // adds to its expert's score.
+    const bool ok = lane < K && myid != kNone;
+    const float qk = ok ? expf(myv - m) : 0.f;
+    float qs = qk;
+    if (a.router_norm != BASE_ROUTER_NORM_TOPK) {   // plain softmax: the denominator runs over all experts
+      qs = 0.f;
 #pragma unroll
-      for (int i = 0; i < NV; ++i) {
-        q[i] = ((taken >> i) & 1u) ? expf(l[i] - m) : 0.f;
-        qs += q[i];
-      }
-    } else {                                        // ... or over all experts (plain softmax)
-#pragma unroll
-      for (int i = 0; i < NV; ++i) {
-        const float qa = ((avail0 >> i) & 1u) ? expf(l[i] - m) : 0.f;
-        q[i] = ((taken >> i) & 1u) ? qa : 0.f;
-        qs += qa;
-      }
+      for (int i = 0; i < NV; ++i) qs += ((avail0 >> i) & 1u) ? expf(l[i] - m) : 0.f;
     }
     const float S_t = warp_sum(qs);
-    // what a routed pair adds to its expert's score: the method's predicted removal cost (the loop the
-    // compiler sees in the common case), or one of the ablation scores
-    const int rule = a.score_rule;
-    if (rule == BASE_SCORE_PREDICTED) {
+    const float w = (ok && S_t > 0.f) ? qk / S_t : 0.f;
+    // predicted log-energy of the route's expert: entry (myid >> 5) of lane (myid & 31)
+    float shk = 0.f;
 #pragma unroll
-      for (int i = 0; i < NV; ++i) {
-        const int e = lane + 32 * i;
-        if (e < E) {
-          float c = 0.f;
-          if ((taken >> i) & 1u) {
-            const float w = S_t > 0.f ? q[i] / S_t : 0.f;
-            c = w * w * expf(sh[i]);
-          }
-          a.ws.costs[size_t(t) * E + e] = c;
-        }
-      }
-    } else {
-      const int first_id = __shfl_sync(0xffffffffu, myid, 0);   // lane k holds the k-th route
-#pragma unroll 1
-      for (int i = 0; i < NV; ++i) {
-        const int e = lane + 32 * i;
-        if (e < E) {
-          float c = 0.f;
-          if ((taken >> i) & 1u) {
-            const float w = S_t > 0.f ? q[i] / S_t : 0.f;
-            if (rule == BASE_SCORE_WEIGHT_SQ) c = w * w;
-            else if (rule == BASE_SCORE_WEIGHT) c = w;
-            else if (rule == BASE_SCORE_STATIC) c = w * w * expf(a.pred_b[e]);
-            else c = (e == first_id) ? 1.f : 0.f;
-          }
-          a.ws.costs[size_t(t) * E + e] = c;
-        }
-      }
+    for (int i = 0; i < NV; ++i) {
+      const float v = __shfl_sync(0xffffffffu, sh[i], ok ? (myid & 31) : 0);
+      if (ok && (myid >> 5) == i) shk = v;
     }
+    // the method's predicted removal cost, or one of the ablation scores
+    const int rule = a.score_rule;
+    float c = 0.f;
+    if (ok) {
+      if (rule == BASE_SCORE_PREDICTED) c = w * w * expf(shk);
+      else if (rule == BASE_SCORE_WEIGHT_SQ) c = w * w;
+      else if (rule == BASE_SCORE_WEIGHT) c = w;
+      else if (rule == BASE_SCORE_STATIC) c = w * w * expf(a.pred_b[myid]);
+      else c = (lane == 0) ? 1.f : 0.f;   // the token's first choice
+    }
+    // dense row: zeros from the lanes that own the entries, then the routed pairs (the warp barrier
+    // orders the two stores to the same address)
+#pragma unroll
+    for (int i = 0; i < NV; ++i) {
+      const int e = lane + 32 * i;
+      if (e < E) a.ws.costs[size_t(t) * E + e] = 0.f;
+    }
+    __syncwarp();
+    if (ok) a.ws.costs[size_t(t) * E + myid] = c;
     if (lane < K) {
-      const bool ok = myid != kNone;
-      const float w = (ok && S_t > 0.f) ? expf(myv - m) / S_t : 0.f;
       const int idx = t * K + lane;
       a.ws.topk_ids[idx] = ok ? myid : -1;
       a.ws.topk_w[idx] = w;
