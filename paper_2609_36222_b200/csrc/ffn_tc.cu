@@ -19,11 +19,19 @@
 // comes from a tensor map whose box height equals the padded token count of the unit.
 //
 // Both passes run in ONE launch. Work units (all gate/up tiles, then all down tiles) are handed out by
-// a global ticket; a down unit waits (bounded) on a per-segment counter of finished gate/up tiles.
-// Because gate/up units never wait and are all taken before any down unit, the scheme cannot
-// deadlock as long as the grid is co-resident (it is: at most one CTA per SM). The gather of the
-// token inputs into expert-sorted order is done by the epilogue warps while the first weight boxes
-// are already in flight.
+// a global ticket; a down unit waits (bounded) on a counter of finished gate/up tiles (per segment, or
+// per expert and K chunk). Because gate/up units never wait on other units and are all taken before
+// any down unit, the scheme cannot deadlock as long as the grid is co-resident (it is: at most one
+// CTA per SM).
+//
+// Batches of at most 128 tokens (one token tile) run the gate/up pass densely: the token operand is
+// the layer input itself, all tokens, read in place, and only the rows of tokens routed to the expert
+// are stored. Such a unit depends on nothing but its expert id, so the kernel starts on the early
+// expert list that the routing kernel publishes while it is still running: CTA c owns gate/up unit
+// c and polls its own list entry; everything that needs the dispatch (the epilogue's row look-up,
+// units past the early list, the down pass) waits for the end of the routing kernel through the
+// programmatic-launch dependency. Larger batches gather the token rows into expert-sorted order
+// (epilogue warps, while the first weight boxes are already in flight) and use per-expert token tiles.
 //
 // Every wait is bounded: on expiry the CTA raises an abort flag, all roles leave their loops, TMEM
 // is freed and BASE_DEV_WAIT_EXPIRED is OR-ed into the status word.

@@ -261,10 +261,15 @@ cudaError_t launch_route_scores(const void* hidden, const void* router_w, const 
 //   -- cluster barrier --
 //   2  every CTA: D[u] = sum_t c[t,u] in a fixed order                              (Sec. 3.4)
 //   3  every CTA: top-M of D by rank counting -> its own copy of the active mask    (Sec. 3.5)
+//      CTA 0: the early expert list for the FFN kernel (selected experts that are certain to be
+//      dispatched), published with one release store as soon as the selection stands
 //      per token: K highest-ranked experts inside the active set, gate = q / S      (Sec. 3.5)
 //   -- cluster barrier --
 //   4  every CTA: tokens dispatched to each expert in token order, offsets by a scan of the counts,
 //      the row of every routed pair in the expert-sorted buffers.
+// Before stage 1 the last CTA clears the FFN kernel's scheduling counters and only then lets that
+// kernel launch; everything up to the early list is on the critical path of the step (the FFN
+// kernel starts streaming 0.8 us after the list appears), the rest runs under its weight stream.
 // Work that needs all tokens (2, 3a, 4) is repeated by every CTA instead of being shared, which
 // leaves two cluster barriers in the whole kernel. Everything is written for short dependent
 // chains: loads are issued in batches, the arg-max is two warp reductions, loop bounds that the
