@@ -132,6 +132,15 @@ typedef struct {
   int ffn_impl;             /* 0: default (tensor-core streaming kernels); 1: simple CUDA-core kernels */
   int score_rule;           /* BASE_SCORE_*: what a routed pair contributes to its expert's batch score */
   int router_norm;          /* BASE_ROUTER_NORM_*: denominator of the router weights w (and of the paper-rule gates) */
+  int expert_first;         /* expert-parallel shard (no counterpart in the paper, which runs on one GPU): when */
+  int expert_count;         /* expert_count > 0, only routed pairs whose expert lies in [expert_first,
+                               expert_first + expert_count) are executed and `out` is this shard's partial sum.
+                               Selection, routes and gates are computed for all experts (identically on every
+                               shard); n_dispatched and expert_counts report the shard's own experts; the
+                               weight arrays are still indexed by the global expert id, but only the rows of the
+                               shard's experts are ever read (the rest of the address range needs no physical
+                               memory behind it). Summing `out` over a partition of the experts
+                               (an all-reduce across ranks; fp32 output recommended) gives the layer's output. */
 } base_layer_options;
 
 /* Bytes of device workspace base_moe_decode_layer needs for up to T_max tokens (0 on bad shape). */

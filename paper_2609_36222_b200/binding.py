@@ -52,7 +52,7 @@ class LayerDebug(C.Structure):
 
 class LayerOptions(C.Structure):
     _fields_ = [("gate_rule", C.c_int), ("fill_rule", C.c_int), ("out_is_fp32", C.c_int), ("ffn_impl", C.c_int),
-                ("score_rule", C.c_int), ("router_norm", C.c_int)]
+                ("score_rule", C.c_int), ("router_norm", C.c_int), ("expert_first", C.c_int), ("expert_count", C.c_int)]
 
 
 class BaseError(RuntimeError):
@@ -201,7 +201,7 @@ def alloc_workspace(nbytes, device):
 
 def base_moe_decode_layer(shape, weights, hidden, budget, out, workspace, router_logits=None, forced_mask=None,
                           gate_rule=GATE_PAPER, fill_rule=FILL_BACKFILL, ffn_impl=FFN_DEFAULT, debug=None,
-                          stream=None, score_rule=SCORE_PREDICTED, router_norm=ROUTER_NORM_TOPK):
+                          stream=None, score_rule=SCORE_PREDICTED, router_norm=ROUTER_NORM_TOPK, expert_range=None):
     """shape: (d, E, K, I); weights: LayerWeights; out: [T,d] bf16 or fp32 tensor (written in place)."""
     d, E, K, I = shape
     T = hidden.shape[0]
@@ -211,7 +211,9 @@ def base_moe_decode_layer(shape, weights, hidden, budget, out, workspace, router
         assert router_logits.dtype == torch.float32 and tuple(router_logits.shape) == (T, E)
     if forced_mask is not None:
         assert forced_mask.dtype == torch.uint8 and forced_mask.numel() == E
-    opt = LayerOptions(gate_rule, fill_rule, 1 if out.dtype == torch.float32 else 0, ffn_impl, score_rule, router_norm)
+    first, count = expert_range if expert_range is not None else (0, 0)   # expert-parallel shard [first, first + count)
+    opt = LayerOptions(gate_rule, fill_rule, 1 if out.dtype == torch.float32 else 0, ffn_impl, score_rule, router_norm,
+                       first, count)
     _check(lib().base_moe_decode_layer(C.byref(LayerShape(d, E, K, I)), C.byref(weights), _ptr(hidden),
                                        _ptr(router_logits), T, budget, _ptr(forced_mask), _ptr(out), C.byref(opt),
                                        C.byref(debug) if debug is not None else None, _ptr(workspace),

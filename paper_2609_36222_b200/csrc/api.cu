@@ -85,6 +85,8 @@ int enqueue_routing(const LayerCall& c, const Workspace& ws, cudaStream_t st, in
   ra.fill_rule = c.opt.fill_rule;
   ra.score_rule = c.opt.score_rule;
   ra.router_norm = c.opt.router_norm;
+  ra.expert_first = c.opt.expert_count > 0 ? c.opt.expert_first : 0;
+  ra.expert_end = c.opt.expert_count > 0 ? c.opt.expert_first + c.opt.expert_count : s.E;
   ra.ffn_first_ticket = c.opt.ffn_impl == 1 ? 0 : ffn_tc_static_units(s, c.T, c.budget, ws);
   ra.ws = ws;
   ra.dbg = c.dbg;
@@ -142,6 +144,8 @@ int check_layer_args(const base_layer_shape* shape, const base_layer_weights* w,
     if (opt->ffn_impl != 0 && opt->ffn_impl != 1) return BASE_ERR_INVALID_ARG;
     if (opt->score_rule < BASE_SCORE_PREDICTED || opt->score_rule > BASE_SCORE_TOP1_UNION) return BASE_ERR_INVALID_ARG;
     if (opt->router_norm != BASE_ROUTER_NORM_TOPK && opt->router_norm != BASE_ROUTER_NORM_ALL) return BASE_ERR_INVALID_ARG;
+    if (opt->expert_count < 0 || (opt->expert_count > 0 && (opt->expert_first < 0 || opt->expert_first + opt->expert_count > shape->E)))
+      return BASE_ERR_INVALID_ARG;
   }
   return BASE_OK;
 }

@@ -180,6 +180,7 @@ struct RoutingArgs {
   const uint8_t* forced_mask; // or nullptr
   const __nv_bfloat16* hidden; // [T,d] token inputs (gathered into expert-sorted order)
   int T, E, K, M, d, gate_rule, fill_rule, max_segs, score_rule, router_norm;
+  int expert_first, expert_end;   // expert-parallel shard: only routes to experts in [first, end) are dispatched
   int ffn_first_ticket;       // units the FFN kernel's CTAs take statically; the ticket counter starts here
   Workspace ws;
   base_layer_debug dbg;       // zero-initialised when the caller passed none

@@ -520,7 +520,7 @@ __global__ void __launch_bounds__(kRoutingThreads) routing_kernel(RoutingArgs a)
   if (cta == 0) {
     const bool eligible = !a.forced_mask && s_status == 0;
     const int e = threadIdx.x;   // E <= kRoutingThreads
-    const bool early = eligible && e < E && s_mask[e] != 0 && s_raw[e] > 0.f;
+    const bool early = eligible && e < E && s_mask[e] != 0 && s_raw[e] > 0.f && e >= a.expert_first && e < a.expert_end;
     const uint32_t bal = __ballot_sync(0xffffffffu, early);
     if (lane == 0) s_wsum[warp] = __popc(bal);
     if (e < E) s_early[e] = early;
@@ -626,7 +626,10 @@ __global__ void __launch_bounds__(kRoutingThreads) routing_kernel(RoutingArgs a)
   // popcounts of these bitmaps, so each expert's rows are in token order.
   const int n_chunks = (T + 31) >> 5;
   for (int i = threadIdx.x; i < S; i += kRoutingThreads) {
-    const int e = a.ws.exec_ids[i];
+    // an expert-parallel shard dispatches only the routes of its own experts; the others keep their
+    // place in exec_ids but get no row
+    const int e_all = a.ws.exec_ids[i];
+    const int e = (e_all >= a.expert_first && e_all < a.expert_end) ? e_all : -1;
     s_eids[i] = e;
     if (e >= 0) {
       const int t = i / K;

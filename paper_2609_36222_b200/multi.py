@@ -54,3 +54,18 @@ def whole_job_us_per_step(ms_per_step_max: float, world: int) -> float:
     """Whole-job figure of the time-like metric: the job completes `world` layer steps (one per
     rank) in the slowest rank's step time."""
     return ms_per_step_max * 1e3 / max(world, 1)
+
+
+def expert_shard(rank: int, world: int, E: int):
+    """Contiguous expert range (first, count) of a rank under expert parallelism; the ranges partition [0, E)."""
+    base, extra = divmod(E, world)
+    first = rank * base + min(rank, extra)
+    return first, base + (1 if rank < extra else 0)
+
+
+def all_reduce_partial_outputs(out, dist):
+    """Sum of the shards' partial layer outputs (the one exchange step of expert parallelism). `out` is the
+    tensor a rank's call wrote with its `expert_range`; with one rank nothing is exchanged."""
+    if dist is not None:
+        dist.all_reduce(out, op=dist.ReduceOp.SUM)
+    return out

@@ -121,6 +121,39 @@ def test_other_model_shapes(E, K, T):
     check_layer(host, dl, 8, router_norm=B.ROUTER_NORM_ALL, gate_rule=B.GATE_RENORM)
 
 
+@pytest.mark.parametrize("name,M,world", [("qwen3", 32, 2), ("qwen3", 32, 8), ("tiny", 6, 3), ("mixtral", 4, 2)])
+def test_expert_parallel_shards_sum_to_the_layer(layers, name, M, world):
+    """Expert parallelism emulated on one GPU: the layer is run once per shard (each executes only the routed
+    pairs of its own experts) and the partial outputs are added, which is what the all-reduce across ranks
+    does. Routes and gates must be the same in every shard; the sum must match the oracle and the unsharded run."""
+    from paper_2609_36222_b200 import multi
+    host, dl = layers(name)
+    cfg = host.cfg
+    logits = O.router_logits(host.z, host.router_w, host.router_bias)
+    ref = O.moe_decode_layer(host.z, logits, host.pred_A, host.pred_b, host.expert_weights, cfg.K, M)
+    hid = bits_to_device(host.hidden_bits, DEV)
+    full = run_gpu(dl, hid, M, logits=logits)
+    total = np.zeros_like(full["y"])
+    n_disp = 0
+    for rank in range(world):
+        first, count = multi.expert_shard(rank, world, cfg.E)
+        part = run_gpu(dl, hid, M, logits=logits, expert_range=(first, count))
+        np.testing.assert_array_equal(part["exec_ids"], full["exec_ids"])
+        np.testing.assert_array_equal(part["exec_gates"], full["exec_gates"])
+        np.testing.assert_array_equal(part["active_mask"], full["active_mask"])
+        local = np.zeros(cfg.E, bool)
+        local[first:first + count] = True
+        assert (part["expert_counts"][~local] == 0).all()
+        np.testing.assert_array_equal(part["expert_counts"][local], full["expert_counts"][local])
+        n_disp += int(part["n_dispatched"][0])
+        total += part["y"]
+    assert n_disp == full["n_dispatched"][0] == ref["n_dispatched"]
+    scale = np.abs(ref["y"]).max()
+    assert np.abs(total - full["y"]).max() <= 1e-5 * scale            # same products, another order of the fp32 sums
+    if set(np.nonzero(full["active_mask"])[0]) == set(ref["selected"].tolist()):
+        assert np.abs(total - ref["y"]).max() <= 6e-3 * scale
+
+
 # ------------------------------------------------------------------------------- edge cases
 
 @pytest.mark.parametrize("T", [1, 5, 33, 130, 256])

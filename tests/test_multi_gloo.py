@@ -54,3 +54,47 @@ def test_single_process_defaults(monkeypatch):
     assert multi.init_process_group("gloo") is None
     assert multi.max_over_ranks(3.5, None) == 3.5
     assert multi.replica_layer_ids(2, 2) == [2000, 2001]
+
+
+def _ep_worker(rank, world, port, out):
+    """Expert parallelism on CPU: every rank combines only its shard's routed pairs of the ORACLE layer (the
+    device kernels are covered on the GPU); the all-reduce of the partial outputs must give the full layer."""
+    import numpy as np
+    from oracle import base_oracle as O
+    os.environ.update(RANK=str(rank), WORLD_SIZE=str(world), LOCAL_RANK=str(rank),
+                      MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist = multi.init_process_group("gloo")
+    r = np.random.default_rng(5)                      # same inputs on every rank (replicated activations)
+    T, d, E, K, I, M = 6, 16, 10, 3, 8, 5
+    z = r.standard_normal((T, d))
+    logits = r.standard_normal((T, E)).astype(np.float32)
+    A, b = 0.1 * r.standard_normal((E, d)), 0.1 * r.standard_normal(E)
+    W = [(r.standard_normal((I, d)), r.standard_normal((I, d)), r.standard_normal((d, I))) for _ in range(E)]
+    full = O.moe_decode_layer(z, logits, A, b, lambda u: W[u], K, M)
+    first, count = multi.expert_shard(rank, world, E)
+    ids = np.where((full["exec_ids"] >= first) & (full["exec_ids"] < first + count), full["exec_ids"], -1)
+    y_part, _ = O.execute(z, ids, full["exec_gates"], lambda u: W[u])
+    t = torch.from_numpy(np.ascontiguousarray(y_part))
+    multi.all_reduce_partial_outputs(t, dist)
+    out[rank] = (first, count, float(np.abs(t.numpy() - full["y"]).max()), float(np.abs(full["y"]).max()))
+    dist.destroy_process_group()
+
+
+def test_expert_parallel_partial_outputs_sum_to_the_layer():
+    world, port = 2, _free_port()
+    with mp.Manager() as m:
+        out = m.dict()
+        mp.spawn(_ep_worker, args=(world, port, out), nprocs=world, join=True)
+        res = dict(out)
+    assert [res[r][:2] for r in (0, 1)] == [(0, 5), (5, 5)]
+    for r in (0, 1):
+        assert res[r][2] <= 1e-12 * res[r][3]
+
+
+def test_expert_shards_partition_the_experts():
+    for E in (8, 60, 128, 7):
+        for world in (1, 2, 3, 8):
+            shards = [multi.expert_shard(r, world, E) for r in range(world)]
+            covered = [e for f, c in shards for e in range(f, f + c)]
+            assert covered == list(range(E))
+            assert max(c for _, c in shards) - min(c for _, c in shards) <= 1
