@@ -251,6 +251,18 @@ int base_true_removal_costs(const base_layer_shape* shape, const base_layer_weig
                             int32_t* topk_ids, float* topk_w, void* workspace, size_t workspace_bytes, void* stream);
 int base_energy_retained(const float* true_scores, const uint8_t* active_mask, int E, int budget, float* out,
                          void* stream);
+/*
+ * Exact error of an active set against its additive estimate (Eq. error_decomposition): the layer is run
+ * with every original route executed, and for the routes whose expert is NOT in active_mask [E] the
+ * contributions a_{t,u} = w_{t,u} E_u(z_t) are summed per token. out[0] = E(A) = sum_t ||sum_u a_{t,u}||^2
+ * (the squared distance between the full layer output and the output with those experts deleted, no
+ * replacement), out[1] = the individual part sum_t sum_u ||a_{t,u}||^2 (= the sum of the true scores D*_u
+ * of the omitted experts), out[2] = their difference, the cross terms. Arguments, workspace and errors as
+ * for base_true_removal_costs.
+ */
+int base_exact_removal_error(const base_layer_shape* shape, const base_layer_weights* weights, const void* hidden_bf16,
+                             const float* router_logits, int T, const uint8_t* active_mask, float* out,
+                             void* workspace, size_t workspace_bytes, void* stream);
 
 /*
  * Offline calibration of the predictor on the device (App. Calibration Details): streaming

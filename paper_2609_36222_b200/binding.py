@@ -28,7 +28,7 @@ EXPORTS = (
     "base_predict_costs", "base_aggregate_select", "base_moe_decode_layer_workspace_bytes",
     "base_moe_decode_layer", "base_moe_decode_layer_noalloc", "base_moe_decode_layer_host_workspace_bytes", "base_moe_decode_layer_host",
     "base_moe_decode_stack_workspace_bytes", "base_moe_decode_stack", "base_profile_events",
-    "base_last_launch_count", "base_true_removal_costs", "base_energy_retained",
+    "base_last_launch_count", "base_true_removal_costs", "base_energy_retained", "base_exact_removal_error",
     "base_calib_state_bytes", "base_calib_workspace_bytes", "base_calib_reset", "base_calib_accumulate",
     "base_calib_solve", "base_calib_accumulate_correction", "base_calib_finalize",
     "base_status_string", "base_last_cuda_error",
@@ -90,6 +90,8 @@ def lib():
     L.base_true_removal_costs.argtypes = [C.POINTER(LayerShape), C.POINTER(LayerWeights), vp, vp, ip, vp, vp, vp, vp,
                                           vp, C.c_size_t, vp]
     L.base_energy_retained.argtypes = [vp, vp, ip, ip, vp, vp]
+    L.base_exact_removal_error.argtypes = [C.POINTER(LayerShape), C.POINTER(LayerWeights), vp, vp, ip, vp, vp, vp,
+                                           C.c_size_t, vp]
     L.base_calib_state_bytes.argtypes = [C.POINTER(LayerShape)]
     L.base_calib_state_bytes.restype = C.c_size_t
     L.base_calib_workspace_bytes.argtypes = [C.POINTER(LayerShape), ip]
@@ -299,6 +301,17 @@ def base_true_removal_costs(shape, weights, hidden, workspace, router_logits=Non
                                          _ptr(router_logits), T, _ptr(true_costs), _ptr(pair_energy), _ptr(topk_ids),
                                          _ptr(topk_w), _ptr(workspace), workspace.numel(), _stream(stream)))
     return true_costs, pair_energy, topk_ids, topk_w
+
+
+def base_exact_removal_error(shape, weights, hidden, active_mask, workspace, router_logits=None, stream=None):
+    """Returns a 3-element tensor: exact error E(A), its individual part, the cross terms (Eq. error_decomposition)."""
+    d, E, K, I = shape
+    assert hidden.dtype == torch.bfloat16 and active_mask.dtype == torch.uint8 and active_mask.numel() == E
+    out = torch.empty(3, dtype=torch.float32, device=hidden.device)
+    _check(lib().base_exact_removal_error(C.byref(LayerShape(d, E, K, I)), C.byref(weights), _ptr(hidden),
+                                          _ptr(router_logits), hidden.shape[0], _ptr(active_mask), _ptr(out),
+                                          _ptr(workspace), workspace.numel(), _stream(stream)))
+    return out
 
 
 def base_energy_retained(true_scores, active_mask, budget, stream=None):

@@ -295,6 +295,35 @@ int base_true_removal_costs(const base_layer_shape* shape, const base_layer_weig
   return BASE_OK;
 }
 
+int base_exact_removal_error(const base_layer_shape* shape, const base_layer_weights* weights, const void* hidden_bf16,
+                             const float* router_logits, int T, const uint8_t* active_mask, float* out,
+                             void* workspace, size_t workspace_bytes, void* stream) {
+  int rc = check_shape(shape, T);
+  if (rc != BASE_OK) return rc;
+  rc = check_layer_args(shape, weights, hidden_bf16, router_logits, T, shape->E, nullptr);
+  if (rc != BASE_OK) return rc;
+  if (!active_mask || !out || !workspace || (reinterpret_cast<uintptr_t>(workspace) & 1023u)) return BASE_ERR_INVALID_ARG;
+  Workspace ws = carve_workspace(workspace, *shape, T);
+  if (ws.bytes > workspace_bytes) return BASE_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  LayerCall c{};
+  c.shape = shape;
+  c.w = weights;
+  c.hidden = hidden_bf16;
+  c.router_logits = router_logits;
+  c.T = T;
+  c.budget = shape->E;   // every original route is executed
+  c.out = ws.x_next;     // the combined output is not wanted
+  int launches = 0, n_split = 1;
+  rc = enqueue_layer(c, ws, st, &launches, &n_split);
+  if (rc != BASE_OK) return rc;
+  // per-token partial results live in the cost matrix of the workspace, which the layer no longer needs
+  cudaError_t e = launch_exact_error(ws, n_split, active_mask, ws.costs, out, T, shape->K, shape->d, st);
+  if (e != cudaSuccess) return cuda_fail(e);
+  g_last_launches = launches + 2;
+  return BASE_OK;
+}
+
 int base_energy_retained(const float* true_scores, const uint8_t* active_mask, int E, int budget, float* out,
                          void* stream) {
   if (!true_scores || !active_mask || !out || E <= 0 || budget <= 0) return BASE_ERR_INVALID_ARG;

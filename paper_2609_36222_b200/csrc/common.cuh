@@ -200,6 +200,8 @@ cudaError_t launch_combine(const Workspace& ws, const void* hidden, void* out, i
 
 cudaError_t launch_pair_energy(const Workspace& ws, int n_split, float* true_costs, float* pair_energy, int T, int E,
                                int K, int d, cudaStream_t st);
+cudaError_t launch_exact_error(const Workspace& ws, int n_split, const uint8_t* mask, float* per_token, float* out, int T,
+                               int K, int d, cudaStream_t st);
 cudaError_t launch_energy_retained(const float* scores, const uint8_t* mask, int E, int budget, float* out,
                                    cudaStream_t st);
 

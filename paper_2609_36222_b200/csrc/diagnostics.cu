@@ -1,6 +1,7 @@
 // Selection-quality diagnostics on the device: true removal costs of routed pairs
 // (Eq. individual_expert_damage) from the per-pair expert outputs that the layer leaves in its
-// workspace, and the retained-energy ratio (Eq. energy_retained).
+// workspace, the exact error of an active set with its individual and cross parts
+// (Eq. error_decomposition), and the retained-energy ratio (Eq. energy_retained).
 #include "common.cuh"
 
 namespace base {
@@ -59,6 +60,94 @@ cudaError_t launch_pair_energy(const Workspace& ws, int n_split, float* true_cos
                     ws.ypair_stride, static_cast<const int32_t*>(ws.exec_ids),
                     static_cast<const float*>(ws.exec_gates), static_cast<const int32_t*>(ws.token_slot), true_costs,
                     pair_energy, E, K, d);
+}
+
+// Exact error of serving the batch with active set A and no replacement (Eq. error_decomposition):
+// per token the omitted contributions a_{t,u} = w_{t,u} E_u(z_t), u in R_t \ A, are added and squared,
+// E(A) = sum_t || sum_u a_{t,u} ||^2, next to the individual part sum_t sum_u ||a_{t,u}||^2; the cross
+// terms are their difference. One CTA per token writes its two numbers; a second kernel adds them in
+// token order.
+__global__ void __launch_bounds__(256) exact_error_token_kernel(const float* __restrict__ ypair, int n_split,
+                                                                size_t split_stride,
+                                                                const int32_t* __restrict__ exec_ids,
+                                                                const float* __restrict__ exec_gates,
+                                                                const int32_t* __restrict__ token_slot,
+                                                                const uint8_t* __restrict__ mask, int K, int d,
+                                                                float* __restrict__ per_token) {
+  __shared__ int s_slot[kMaxK];
+  __shared__ float s_gate[kMaxK];
+  __shared__ float s_tot[8], s_ind[8];
+  const int t = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  pdl_launch_dependents();
+  pdl_wait();
+  if (threadIdx.x < kMaxK) {
+    int slot = -1;
+    float g = 0.f;
+    if (int(threadIdx.x) < K) {
+      const int e = exec_ids[t * K + threadIdx.x];
+      if (e >= 0 && !mask[e]) {   // an omitted route
+        slot = token_slot[t * K + threadIdx.x];
+        g = exec_gates[t * K + threadIdx.x];
+      }
+    }
+    s_slot[threadIdx.x] = slot;
+    s_gate[threadIdx.x] = g;
+  }
+  __syncthreads();
+  float tot = 0.f, ind = 0.f;
+  for (int c = threadIdx.x; c < d; c += 256) {
+    float v = 0.f;
+    for (int k = 0; k < K; ++k) {
+      const int slot = s_slot[k];
+      if (slot < 0) continue;
+      float y = ypair[size_t(slot) * d + c];
+      for (int s = 1; s < n_split; ++s) y += ypair[size_t(s) * split_stride + size_t(slot) * d + c];
+      const float a = s_gate[k] * y;
+      v += a;
+      ind = fmaf(a, a, ind);
+    }
+    tot = fmaf(v, v, tot);
+  }
+  tot = warp_sum(tot);
+  ind = warp_sum(ind);
+  if (lane == 0) {
+    s_tot[warp] = tot;
+    s_ind[warp] = ind;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float a = 0.f, b = 0.f;
+    for (int w = 0; w < 8; ++w) {
+      a += s_tot[w];
+      b += s_ind[w];
+    }
+    per_token[2 * t] = a;
+    per_token[2 * t + 1] = b;
+  }
+}
+
+__global__ void exact_error_sum_kernel(const float* __restrict__ per_token, int T, float* __restrict__ out) {
+  pdl_launch_dependents();
+  pdl_wait();
+  if (threadIdx.x != 0) return;
+  double tot = 0.0, ind = 0.0;
+  for (int t = 0; t < T; ++t) {
+    tot += double(per_token[2 * t]);
+    ind += double(per_token[2 * t + 1]);
+  }
+  out[0] = float(tot);
+  out[1] = float(ind);
+  out[2] = float(tot - ind);
+}
+
+cudaError_t launch_exact_error(const Workspace& ws, int n_split, const uint8_t* mask, float* per_token, float* out, int T,
+                               int K, int d, cudaStream_t st) {
+  cudaError_t e = launch_pdl(exact_error_token_kernel, dim3(T), dim3(256), 0, st, 1, static_cast<const float*>(ws.ypair),
+                             n_split, ws.ypair_stride, static_cast<const int32_t*>(ws.exec_ids),
+                             static_cast<const float*>(ws.exec_gates), static_cast<const int32_t*>(ws.token_slot), mask, K,
+                             d, per_token);
+  if (e != cudaSuccess) return e;
+  return launch_pdl(exact_error_sum_kernel, dim3(1), dim3(32), 0, st, 1, static_cast<const float*>(per_token), T, out);
 }
 
 // Retained energy of an active set: one CTA. An expert belongs to the oracle set A* when fewer than

@@ -86,3 +86,33 @@ def test_true_costs_error_codes():
     m = torch.zeros(4, dtype=torch.uint8, device=DEV)
     with pytest.raises(B.BaseError, match="invalid"):
         B.base_energy_retained(s, m, 0)
+
+
+@pytest.mark.parametrize("name,T", [("tiny", 8), ("mid", 32)])
+def test_exact_error_decomposition_matches_oracle(name, T):
+    """E(A), its individual part and the cross terms (Eq. error_decomposition) for BASE's own selection and for
+    two degenerate masks; the individual part must also equal the true scores of the omitted experts."""
+    cfg = wl.CONFIGS[name]
+    host = HostLayer(cfg, T=T)
+    dl = device_layer_from_host(host, DEV)
+    logits = O.router_logits(host.z, host.router_w, host.router_bias)
+    _, R, _, _, w = O.route_topk(logits, cfg.K)
+    a = O.contributions(host.z, R, w, host.expert_weights)
+    D = O.true_removal_cost(a, R, cfg.E)
+    hid = bits_to_device(host.hidden_bits, DEV)
+    lg = torch.from_numpy(logits).to(DEV)
+    M = cfg.budgets[0]
+    base_mask = O.moe_decode_layer(host.z, logits, host.pred_A, host.pred_b, host.expert_weights, cfg.K, M)["mask"]
+    every_other = (np.arange(cfg.E) % 2 == 0).astype(np.uint8)
+    for mask in (base_mask.astype(np.uint8), every_other, np.ones(cfg.E, np.uint8), np.zeros(cfg.E, np.uint8)):
+        got = B.base_exact_removal_error(dl.shape, dl.weights, hid, torch.from_numpy(mask).to(DEV), dl.workspace,
+                                         router_logits=lg).cpu().numpy().astype(np.float64)
+        total, indiv, cross = O.exact_error(a, R, mask)
+        scale = max(indiv, 1e-30)
+        assert abs(got[0] - total) <= ENERGY_RTOL * scale
+        assert abs(got[1] - indiv) <= ENERGY_RTOL * scale
+        assert abs(got[2] - cross) <= 2 * ENERGY_RTOL * scale
+        assert abs(got[1] - D[mask == 0].sum()) <= ENERGY_RTOL * scale          # additive estimate: sum of D*_u
+        assert got[0] >= 0 and abs(got[0] - got[1] - got[2]) <= 1e-5 * max(got[0], scale)
+        if mask.all():
+            assert (got == 0).all()
