@@ -429,6 +429,7 @@ def run_ours(args, cfg, T, M):
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
+    return line
 
 
 def run_calibration(args, cfg, T):
@@ -507,6 +508,8 @@ def main():
     ap.add_argument("--no-dense", action="store_true", help="skip the unlimited-budget run")
     ap.add_argument("--profile", action="store_true",
                     help="only the warm-up and the timed steps (for a short run under a profiler)")
+    ap.add_argument("--sweep", action="store_true",
+                    help="one line per budget of the workload, then the linear fit of step time against dispatched experts")
     ap.add_argument("--single-step-graphs", action="store_true",
                     help="replay one graph per step instead of one graph per round of weight replicas")
     ap.add_argument("--bias-scale", type=float, default=1.0,
@@ -520,7 +523,25 @@ def main():
     cfg = wl.CONFIGS[args.workload]
     T = args.batch or cfg.T
     M = args.budget
-    if args.calib:
+    if args.sweep:
+        # extra lines (one per budget of the workload) and the least-squares fit t = a + b * dispatched,
+        # the analogue of the paper's Table latency_budget_regression
+        args.no_cpu = True
+        pts = []
+        for m in cfg.budgets:
+            line = run_ours(args, cfg, T, m)
+            if line is not None:
+                pts.append((line["config"]["n_dispatched_mean"], line["value"]))
+        if len(pts) >= 2 and len({p[0] for p in pts}) >= 2:
+            x, y = np.array([p[0] for p in pts]), np.array([p[1] for p in pts])
+            A = np.vstack([np.ones_like(x), x]).T
+            coef = np.linalg.lstsq(A, y, rcond=None)[0]
+            pred = A @ coef
+            r2 = 1.0 - float(((y - pred) ** 2).sum() / max(((y - y.mean()) ** 2).sum(), 1e-30))
+            print(json.dumps({"fit": "us_per_step = a + b * n_dispatched", "a_us": float(coef[0]),
+                              "b_us_per_expert": float(coef[1]), "r2": r2, "points": pts,
+                              "expert_bytes": cfg.expert_bytes}))
+    elif args.calib:
         run_calibration(args, cfg, args.batch or 1024)
     elif args.impl == "reference":
         run_reference(args, cfg, T, M)
