@@ -52,7 +52,8 @@ enum {                             /* bits of the device status word */
 };
 
 enum { BASE_GATE_PAPER = 0,        /* Sec. 3.5: original top-K denominator (gates may sum to < 1) */
-       BASE_GATE_RENORM = 1 };     /* renormalise over the executed experts (OEA-style variant) */
+       BASE_GATE_RENORM = 1,       /* renormalise over the executed experts (OEA-style variant) */
+       BASE_GATE_ONE = 2 };        /* every executed expert enters with weight 1 */
 enum { BASE_SCORE_PREDICTED = 0,   /* Eq. log_energy_predictor: sum of w^2 exp(a.z/|z| + b) (the method) */
        BASE_SCORE_WEIGHT_SQ = 1,   /* squared router-weight sum, sum of w^2   (App. Selection-Rule Ablation) */
        BASE_SCORE_WEIGHT = 2,      /* router-weight sum, sum of w */
@@ -132,6 +133,10 @@ typedef struct {
   int ffn_impl;             /* 0: default (tensor-core streaming kernels); 1: simple CUDA-core kernels */
   int score_rule;           /* BASE_SCORE_*: what a routed pair contributes to its expert's batch score */
   int router_norm;          /* BASE_ROUTER_NORM_*: denominator of the router weights w (and of the paper-rule gates) */
+  int accumulate_out;       /* 1: the result is ADDED to what `out` already holds instead of overwriting it. With
+                               BASE_GATE_ONE, K = E = budget = the number of shared experts and any logits, a
+                               second call adds always-on shared experts (Sec. 3.1 leaves them out of the
+                               selection) to a layer's output: out += sum_s E_s(z_t). */
   int expert_first;         /* expert-parallel shard (no counterpart in the paper, which runs on one GPU): when */
   int expert_count;         /* expert_count > 0, only routed pairs whose expert lies in [expert_first,
                                expert_first + expert_count) are executed and `out` is this shard's partial sum.

@@ -25,6 +25,7 @@ import numpy as np
 
 GATE_RULE_PAPER = 0       # Sec. 3.5: denominator from the token's ORIGINAL top-K
 GATE_RULE_RENORM = 1      # OEA-style: renormalise over the executed experts
+GATE_RULE_ONE = 2         # every executed expert enters with weight 1 (always-on shared experts, Sec. 3.1)
 FILL_BACKFILL = 0         # Sec. 3.5: next-preferred experts inside the active set
 FILL_DROP = 1             # fill-rule ablation: unavailable routes are simply removed
 ROUTER_NORM_TOPK = 0      # router weights renormalised over the token's top-K
@@ -137,7 +138,7 @@ def restrict_routes(order, R, q, S, mask, K, gate_rule=GATE_RULE_PAPER, fill=FIL
 
     Backfill: the token's K highest-ranked experts inside the active set. Gate of an executed expert
     is its own router score q over the ORIGINAL top-K denominator S_t (paper rule), or over the sum
-    of the executed scores (renorm rule). Empty slots: id -1, gate 0. Returns (ids [T,K], gates [T,K]).
+    of the executed scores (renorm rule), or simply 1 (the rule for always-on shared experts). Empty slots: id -1, gate 0. Returns (ids [T,K], gates [T,K]).
     """
     T = order.shape[0]
     ids = np.full((T, K), -1, np.int32)
@@ -150,6 +151,9 @@ def restrict_routes(order, R, q, S, mask, K, gate_rule=GATE_RULE_PAPER, fill=FIL
         for k, u in enumerate(kept):
             ids[t, k] = u
             gates[t, k] = q[t, u]
+        if gate_rule == GATE_RULE_ONE:
+            gates[t] = (ids[t] >= 0).astype(np.float64)
+            continue
         den = S[t] if gate_rule == GATE_RULE_PAPER else gates[t].sum()
         if den > 0:
             gates[t] /= den

@@ -17,7 +17,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.environ.get("BASE_MOE_LIB") or os.path.join(_HERE, "libbase_moe.so")
 
 BASE_OK = 0
-GATE_PAPER, GATE_RENORM = 0, 1
+GATE_PAPER, GATE_RENORM, GATE_ONE = 0, 1, 2
 FILL_BACKFILL, FILL_DROP = 0, 1
 FFN_DEFAULT, FFN_SIMPLE = 0, 1
 SCORE_PREDICTED, SCORE_WEIGHT_SQ, SCORE_WEIGHT, SCORE_STATIC, SCORE_TOP1_UNION = 0, 1, 2, 3, 4
@@ -52,7 +52,8 @@ class LayerDebug(C.Structure):
 
 class LayerOptions(C.Structure):
     _fields_ = [("gate_rule", C.c_int), ("fill_rule", C.c_int), ("out_is_fp32", C.c_int), ("ffn_impl", C.c_int),
-                ("score_rule", C.c_int), ("router_norm", C.c_int), ("expert_first", C.c_int), ("expert_count", C.c_int)]
+                ("score_rule", C.c_int), ("router_norm", C.c_int), ("accumulate_out", C.c_int), ("expert_first", C.c_int),
+                ("expert_count", C.c_int)]
 
 
 class BaseError(RuntimeError):
@@ -203,7 +204,7 @@ def alloc_workspace(nbytes, device):
 
 def base_moe_decode_layer(shape, weights, hidden, budget, out, workspace, router_logits=None, forced_mask=None,
                           gate_rule=GATE_PAPER, fill_rule=FILL_BACKFILL, ffn_impl=FFN_DEFAULT, debug=None,
-                          stream=None, score_rule=SCORE_PREDICTED, router_norm=ROUTER_NORM_TOPK, expert_range=None):
+                          stream=None, score_rule=SCORE_PREDICTED, router_norm=ROUTER_NORM_TOPK, expert_range=None, accumulate=False):
     """shape: (d, E, K, I); weights: LayerWeights; out: [T,d] bf16 or fp32 tensor (written in place)."""
     d, E, K, I = shape
     T = hidden.shape[0]
@@ -215,7 +216,7 @@ def base_moe_decode_layer(shape, weights, hidden, budget, out, workspace, router
         assert forced_mask.dtype == torch.uint8 and forced_mask.numel() == E
     first, count = expert_range if expert_range is not None else (0, 0)   # expert-parallel shard [first, first + count)
     opt = LayerOptions(gate_rule, fill_rule, 1 if out.dtype == torch.float32 else 0, ffn_impl, score_rule, router_norm,
-                       first, count)
+                       1 if accumulate else 0, first, count)
     _check(lib().base_moe_decode_layer(C.byref(LayerShape(d, E, K, I)), C.byref(weights), _ptr(hidden),
                                        _ptr(router_logits), T, budget, _ptr(forced_mask), _ptr(out), C.byref(opt),
                                        C.byref(debug) if debug is not None else None, _ptr(workspace),

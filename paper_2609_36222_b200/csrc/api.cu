@@ -119,7 +119,8 @@ int enqueue_layer(const LayerCall& c, const Workspace& ws, cudaStream_t st, int*
   if (e != cudaSuccess) return cuda_fail(e);
   mark(4, st);
 
-  e = launch_combine(ws, c.hidden, c.out, c.opt.out_is_fp32, c.x_next, c.T, s.K, s.d, n_split, st);
+  e = launch_combine(ws, c.hidden, c.out, (c.opt.out_is_fp32 ? 1 : 0) | ((c.opt.accumulate_out && !c.x_next) ? 2 : 0), c.x_next,
+                     c.T, s.K, s.d, n_split, st);
   if (e != cudaSuccess) return cuda_fail(e);
   ++*launches;
   mark(5, st);
@@ -139,7 +140,7 @@ int check_layer_args(const base_layer_shape* shape, const base_layer_weights* w,
     return BASE_ERR_INVALID_ARG;
   if ((!opt || opt->ffn_impl == 0) && shape->d % 128 != 0) return BASE_ERR_UNSUPPORTED;
   if (opt) {
-    if (opt->gate_rule != BASE_GATE_PAPER && opt->gate_rule != BASE_GATE_RENORM) return BASE_ERR_INVALID_ARG;
+    if (opt->gate_rule < BASE_GATE_PAPER || opt->gate_rule > BASE_GATE_ONE) return BASE_ERR_INVALID_ARG;
     if (opt->fill_rule != BASE_FILL_BACKFILL && opt->fill_rule != BASE_FILL_DROP) return BASE_ERR_INVALID_ARG;
     if (opt->ffn_impl != 0 && opt->ffn_impl != 1) return BASE_ERR_INVALID_ARG;
     if (opt->score_rule < BASE_SCORE_PREDICTED || opt->score_rule > BASE_SCORE_TOP1_UNION) return BASE_ERR_INVALID_ARG;

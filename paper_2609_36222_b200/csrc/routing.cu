@@ -608,7 +608,7 @@ __global__ void __launch_bounds__(kRoutingThreads) routing_kernel(RoutingArgs a)
       if (mypos < 0) mypos = __popc(filled) + __popc(~filled & ((1u << lane) - 1u));
       const float den = (a.gate_rule == BASE_GATE_RENORM) ? sumq : S_t;
       const bool ok = myid != kNone;
-      const float g = (ok && den > 0.f) ? myq / den : 0.f;
+      const float g = (a.gate_rule == BASE_GATE_ONE) ? (ok ? 1.f : 0.f) : ((ok && den > 0.f) ? myq / den : 0.f);
       const int idx = t * K + mypos;
       a.ws.exec_ids[idx] = ok ? myid : -1;
       a.ws.exec_gates[idx] = g;
@@ -922,14 +922,31 @@ __global__ void __launch_bounds__(256) combine_out_kernel(const float* __restric
       }
     }
   }
-  if (out_is_fp32) {
-    *reinterpret_cast<float4*>(static_cast<float*>(out) + size_t(t) * d + c) = acc;
+  // out_is_fp32: bit 0 = fp32 output, bit 1 = add to what the output already holds
+  if (out_is_fp32 & 1) {
+    float4* o = reinterpret_cast<float4*>(static_cast<float*>(out) + size_t(t) * d + c);
+    if (out_is_fp32 & 2) {
+      const float4 old = *o;
+      acc.x += old.x;
+      acc.y += old.y;
+      acc.z += old.z;
+      acc.w += old.w;
+    }
+    *o = acc;
   } else {
+    uint2* o = reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(out) + size_t(t) * d + c);
+    if (out_is_fp32 & 2) {
+      const uint2 old = *o;
+      acc.x += __uint_as_float(old.x << 16);
+      acc.y += __uint_as_float(old.x & 0xffff0000u);
+      acc.z += __uint_as_float(old.y << 16);
+      acc.w += __uint_as_float(old.y & 0xffff0000u);
+    }
     __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
     uint2 p;
     p.x = *reinterpret_cast<uint32_t*>(&lo);
     p.y = *reinterpret_cast<uint32_t*>(&hi);
-    *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(out) + size_t(t) * d + c) = p;
+    *o = p;
   }
 }
 

@@ -154,6 +154,32 @@ def test_expert_parallel_shards_sum_to_the_layer(layers, name, M, world):
         assert np.abs(total - ref["y"]).max() <= 6e-3 * scale
 
 
+@pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16])
+def test_shared_experts_added_by_a_second_call(out_dtype):
+    """A layer with always-on shared experts (the paper's other two models, Sec. 4.1; left out of the selection,
+    Sec. 3.1): the routed experts go through BASE, then a second call with the unit gate rule, K = E = budget =
+    number of shared experts and `accumulate` adds sum_s E_s(z_t) to the same output."""
+    T = 48
+    routed = wl.LayerConfig("shared_routed", d=1024, E=64, K=6, I=704, T=T, budgets=(20,))
+    shared = wl.LayerConfig("shared_always", d=1024, E=2, K=2, I=704, T=T, budgets=(2,))
+    hr, hs = HostLayer(routed, T=T), HostLayer(shared, T=T)
+    hs.hidden_bits = hr.hidden_bits                                   # the same tokens
+    dr, ds = device_layer_from_host(hr, DEV), device_layer_from_host(hs, DEV)
+    logits = O.router_logits(hr.z, hr.router_w, hr.router_bias)
+    ref = O.moe_decode_layer(hr.z, logits, hr.pred_A, hr.pred_b, hr.expert_weights, routed.K, 20)
+    want = ref["y"] + sum(O.expert_ffn(hr.z, *hs.expert_weights(u)) for u in range(shared.E))
+    hid = bits_to_device(hr.hidden_bits, DEV)
+    out = torch.full((T, routed.d), float("nan"), dtype=out_dtype, device=DEV)
+    B.base_moe_decode_layer(dr.shape, dr.weights, hid, 20, out, dr.workspace, router_logits=torch.from_numpy(logits).to(DEV))
+    B.base_moe_decode_layer(ds.shape, ds.weights, hid, 2, out, ds.workspace,
+                            router_logits=torch.zeros(T, 2, dtype=torch.float32, device=DEV),
+                            gate_rule=B.GATE_ONE, accumulate=True)
+    torch.cuda.synchronize()
+    got = out.float().cpu().numpy().astype(np.float64)
+    scale = np.abs(want).max()
+    assert np.abs(got - want).max() <= (6e-3 if out_dtype == torch.float32 else 1.6e-2) * scale
+
+
 # ------------------------------------------------------------------------------- edge cases
 
 @pytest.mark.parametrize("T", [1, 5, 33, 130, 256])

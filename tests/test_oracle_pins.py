@@ -141,6 +141,20 @@ def test_gate_rules():
     np.testing.assert_array_equal(ren["exec_ids"], out["exec_ids"])
 
 
+def test_unit_gate_rule_is_a_plain_sum_of_experts():
+    """GATE_RULE_ONE with K = E = M: every token runs every expert with weight 1, i.e. the layer is the plain sum
+    of the experts' outputs (how always-on shared experts, which Sec. 3.1 leaves out of the selection, are added)."""
+    r = np.random.default_rng(21)
+    T, d, E, I = 5, 8, 3, 6
+    z = r.standard_normal((T, d))
+    W = [(r.standard_normal((I, d)), r.standard_normal((I, d)), r.standard_normal((d, I))) for _ in range(E)]
+    logits = r.standard_normal((T, E)).astype(np.float32)            # any logits: the gates ignore them
+    out = O.moe_decode_layer(z, logits, np.zeros((E, d)), np.zeros(E), lambda u: W[u], E, E, gate_rule=O.GATE_RULE_ONE)
+    want = sum(O.expert_ffn(z, *W[u]) for u in range(E))
+    np.testing.assert_allclose(out["y"], want, rtol=1e-12, atol=1e-12)
+    assert (out["exec_gates"] == 1.0).all() and out["n_dispatched"] == E
+
+
 def test_budget_below_topk_leaves_empty_slots():
     z, logits, A, b, ew = make_layer(9, E=8, K=3)
     out = O.moe_decode_layer(z, logits, A, b, ew, 3, 2)
