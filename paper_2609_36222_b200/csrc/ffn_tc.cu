@@ -253,6 +253,7 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true, x_ready = false;
+      const uint64_t pol_w = l2_policy_evict_first();   // weights are read once
       CYC_DECL(c_wait); CYC_DECL(c_issue); CYC_DECL(c_rows); CYC_DECL(c_n); CYC_DECL(c_rows_gu); CYC_DECL(c_units); CYC_DECL(c_t_first); CYC_DECL(c_t_gu_end);
       CYC_T0(t_start);
       // the ticket and the decoding of the next unit are requested one unit ahead, so their memory
@@ -350,16 +351,16 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
           mbar_expect_tx(full, bytes);
           if (gu) {
             if (!p.split_a) {
-              tma_load_4d(sa, &maps1.a, 0, arow, 0, kb, full);      // {elem, row, gate|up, k-block}
+              tma_load_4d_hint(sa, &maps1.a, 0, arow, 0, kb, full, pol_w);      // {elem, row, gate|up, k-block}
             } else {
 #pragma unroll
               for (int j = 0; j < kKbPerStage; ++j) {
-                tma_load_3d(sa + j * kTileABytes, &maps1.a, 0, arow, kb + j, full);
-                tma_load_3d(sa + j * kTileABytes + kTileABytes / 2, &maps1.a2, 0, arow, kb + j, full);
+                tma_load_3d_hint(sa + j * kTileABytes, &maps1.a, 0, arow, kb + j, full, pol_w);
+                tma_load_3d_hint(sa + j * kTileABytes + kTileABytes / 2, &maps1.a2, 0, arow, kb + j, full, pol_w);
               }
             }
           } else {
-            tma_load_3d(sa, &maps2.a, 0, arow, kb, full);            // {elem, row, k-block}
+            tma_load_3d_hint(sa, &maps2.a, 0, arow, kb, full, pol_w);          // {elem, row, k-block}
           }
           if (!b_ready) {
             CYC_T0(t_r);
