@@ -53,6 +53,7 @@ struct LayerCall {
   base_layer_options opt;
   base_layer_debug dbg;
   void* x_next;  // stack wiring output or nullptr
+  const base_layer_weights* next_w = nullptr;  // stack: the layer that runs after this one
 };
 
 // Router + predictor GEMV and the routing kernel of one layer (selection, restricted routes, dispatch lists).
@@ -114,7 +115,10 @@ int enqueue_layer(const LayerCall& c, const Workspace& ws, cudaStream_t st, int*
   if (c.opt.ffn_impl == 1) {
     e = launch_ffn_simple(s, *c.w, ws, st, launches);
   } else {
-    e = launch_ffn_tc(s, *c.w, c.hidden, ws, c.T, c.budget, st, launches, &n_split);
+    // the next layer's router and predictor matrices are known now and needed first thing after this
+    // layer: the FFN kernel asks the L2 for them while it streams
+    const void* ahead[2] = {c.next_w ? c.next_w->router_w : nullptr, c.next_w ? c.next_w->pred_A : nullptr};
+    e = launch_ffn_tc(s, *c.w, c.hidden, ws, c.T, c.budget, ahead, st, launches, &n_split);
   }
   if (e != cudaSuccess) return cuda_fail(e);
   mark(4, st);
@@ -510,6 +514,7 @@ int base_moe_decode_stack(const base_layer_shape* shape, const base_layer_weight
     if (opt) c.opt = *opt;
     if (n_dispatched_per_layer) c.dbg.n_dispatched = n_dispatched_per_layer + l;
     c.x_next = (l == L - 1) ? out : ping[l & 1];
+    c.next_w = (l + 1 < L) ? &h_weights[l + 1] : nullptr;
     int rc = enqueue_layer(c, ws, st, &launches);
     if (rc != BASE_OK) return rc;
     x = c.x_next;

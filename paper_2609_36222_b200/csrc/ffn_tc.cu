@@ -129,6 +129,7 @@ struct FfnParams {
   int kb2;              // down pass: k-blocks per unit = ceil(I/64 / ksplit), even (= gate/up tiles a unit depends on)
   long long* cycles;    // developer aid (-DBASE_FFN_CYCLES)
   int split_a;          // gate/up pass: 1 = gate and up come from two maps (two boxes per k-block)
+  const char* ahead[2]; // [E,d] bf16 matrices of the next layer (router, predictor) to request into the L2, or nullptr
 };
 
 // SwiGLU gate with the hardware exponential and reciprocal (relative error ~1e-6, far below bf16)
@@ -236,6 +237,18 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
   // end of that kernel only when it needs the dispatch itself.
   const int down_units_per_seg = p.tiles2 * (kSplit > 1 ? p.ksplit : 1);
   int n_slots = 0;
+  if (warp == 2 && lane < 2 && p.ahead[lane]) {
+    // The next layer's score kernel starts with these matrices; they are constant, so they can be
+    // requested now: one slice per CTA, fire and forget (the weight stream is evict-first and leaves
+    // them alone).
+    const uint32_t total = uint32_t(p.E) * uint32_t(p.d) * 2u;
+    const uint32_t slice = ((total + gridDim.x - 1) / gridDim.x + 15u) & ~15u;
+    const uint32_t lo = blockIdx.x * slice;
+    if (lo < total) {
+      const uint32_t n = min(slice, total - lo);   // total and slice are multiples of 16 bytes
+      asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p.ahead[lane] + lo), "r"(n) : "memory");
+    }
+  }
   if (!kDense) {
     pdl_wait();
     n_slots = p.counters[kCtrSlots];
@@ -851,7 +864,8 @@ bool tc_map_rows_kblocks(const void* ptr, uint64_t rows, uint64_t cols, uint32_t
 int tc_sm_count() { return sm_count(); }
 
 cudaError_t launch_ffn_tc(const base_layer_shape& s, const base_layer_weights& w, const void* hidden,
-                          const Workspace& ws, int T, int budget, cudaStream_t st, int* launches, int* n_split) {
+                          const Workspace& ws, int T, int budget, const void* const ahead[2], cudaStream_t st,
+                          int* launches, int* n_split) {
   const uint64_t slots = uint64_t(T) * s.K + kRowPad;
   const uint64_t wrows = uint64_t(s.E) * s.I;
   MapSet m1{}, m2{};
@@ -894,6 +908,8 @@ cudaError_t launch_ffn_tc(const base_layer_shape& s, const base_layer_weights& w
   p.E = s.E;
   p.I = s.I;
   p.d = s.d;
+  p.ahead[0] = static_cast<const char*>(ahead[0]);
+  p.ahead[1] = static_cast<const char*>(ahead[1]);
 #ifdef BASE_FFN_CYCLES
   p.cycles = reinterpret_cast<long long*>(ws.x_next);   // scratch that a single-layer call does not use
 #endif
