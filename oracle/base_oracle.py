@@ -323,8 +323,56 @@ def ridge_fit(X, y, lam):
     return a, float(ym - a @ xm)
 
 
+def lambda_grid(n=25, lo=1e-4, hi=1e2):
+    """The ridge penalties tried per expert: n values logarithmically spaced from lo to hi (App. Calibration Details)."""
+    return lo * (hi / lo) ** (np.arange(n, dtype=np.float64) / (n - 1))
+
+
+def ridge_log_evidence(X, y, lambdas):
+    """Log marginal likelihood of each ridge penalty, up to a constant that does not depend on it.
+
+    Model behind the centred ridge of App. Calibration Details: y = X a + b 1 + noise, noise ~ N(0, s2 I),
+    a ~ N(0, (s2 / lam) I), flat prior on the intercept b, noise variance s2 at its maximising value. With
+    G_c = X_c^T X_c, q_c = X_c^T y_c (centred statistics, n pairs, d features) and the eigenvalues theta_i and
+    eigenvectors v_i of G_c -- the one eigendecomposition that serves every penalty --
+
+        r(lam) = y_c.y_c - sum_i (v_i.q_c)^2 / (theta_i + lam)      (= y_c.y_c - q_c^T (G_c + lam I)^-1 q_c)
+        L(lam) = -(n - 1)/2 * log r(lam) - 1/2 * sum_i log(1 + theta_i / lam).
+
+    The paper names the criterion but prints no formula; this is this implementation's reading. r is
+    floored at 1e-12 * y_c.y_c + 1e-300 (an exact fit must not produce log 0). Returns L [len(lambdas)].
+    """
+    X = np.asarray(X, np.float64)
+    y = np.asarray(y, np.float64)
+    n = X.shape[0]
+    Xc = X - X.mean(axis=0)
+    yc = y - y.mean()
+    theta, V = np.linalg.eigh(Xc.T @ Xc)
+    theta = np.maximum(theta, 0.0)
+    proj = (V.T @ (Xc.T @ yc)) ** 2
+    yy = float(yc @ yc)
+    out = np.empty(len(lambdas))
+    for i, lam in enumerate(np.asarray(lambdas, np.float64)):
+        r = max(yy - float((proj / (theta + lam)).sum()), 1e-12 * yy + 1e-300)
+        out[i] = -0.5 * (n - 1) * np.log(r) - 0.5 * float(np.log1p(theta / lam).sum())
+    return out
+
+
+def select_lambda(X, y, lambdas, default_index=None):
+    """Index of the penalty with the largest evidence (the first one on a tie). An expert with fewer than two
+    pairs has no centred statistics to judge by and takes default_index (the middle of the grid if None)."""
+    if default_index is None:
+        default_index = len(lambdas) // 2
+    if np.asarray(X).shape[0] < 2:
+        return default_index
+    return int(np.argmax(ridge_log_evidence(X, y, lambdas)))
+
+
 def fit_predictor(z_calib, logits_calib, expert_weights, K, E, lam=1e-2, eps=1e-12):
     """Fit (a_u, b_u) per expert on routed calibration pairs.
+
+    lam: a fixed ridge penalty, or an array of candidates from which every expert takes the one of largest
+    evidence (select_lambda).
 
     Target s = log(||E_u(z)||^2 + eps) (Sec. 3.4), features z-bar. The intercept is shifted by
     log(mean energy / mean exp(s-hat)) so that the mean predicted energy equals the mean true
@@ -348,7 +396,8 @@ def fit_predictor(z_calib, logits_calib, expert_weights, K, E, lam=1e-2, eps=1e-
         energy = (out * out).sum(axis=1)
         all_energy.append(energy)
         s = np.log(energy + eps)
-        a_u, b_u = ridge_fit(zbar[tt], s, lam)
+        lam_u = lam if np.isscalar(lam) else float(np.asarray(lam)[select_lambda(zbar[tt], s, lam)])
+        a_u, b_u = ridge_fit(zbar[tt], s, lam_u)
         s_hat = zbar[tt] @ a_u + b_u
         b_u += float(np.log(np.mean(energy) / np.mean(np.exp(s_hat))))
         A[u], b[u], fitted[u] = a_u, b_u, True

@@ -348,6 +348,71 @@ def test_ridge_matches_least_squares_and_recovers_planted_model():
     assert norms == sorted(norms, reverse=True)
 
 
+def test_lambda_grid_is_the_papers():
+    g = O.lambda_grid()
+    assert len(g) == 25 and g[0] == pytest.approx(1e-4) and g[-1] == pytest.approx(1e2)
+    np.testing.assert_allclose(g[1:] / g[:-1], 10 ** 0.25, rtol=1e-12)      # logarithmic spacing
+
+
+def test_ridge_evidence_is_the_profiled_gaussian_marginal_density():
+    """The weight-space expression (eigenvalues of the d x d centred Gram matrix) against the function-space
+    definition: the density of the centred targets under N(0, s2 (I + X X^T / lam)), evaluated by scipy and
+    maximised over s2 numerically. Sylvester's determinant identity and Woodbury connect the two."""
+    from scipy.linalg import null_space
+    from scipy.optimize import minimize_scalar
+    from scipy.stats import multivariate_normal
+    r = np.random.default_rng(31)
+    n, d = 12, 5
+    X = r.standard_normal((n, d))
+    y = X @ r.standard_normal(d) + 0.3 * r.standard_normal(n) + 2.0
+    Q = null_space(np.ones((1, n)))                     # orthonormal basis of the complement of the intercept
+    yt, Xt = Q.T @ y, Q.T @ X
+    lambdas = np.array([1e-3, 0.05, 1.0, 7.0, 100.0])
+    L = O.ridge_log_evidence(X, y, lambdas)
+    const = 0.5 * (n - 1) * (np.log(n - 1) - np.log(2 * np.pi) - 1.0)
+    for lam, l_val in zip(lambdas, L):
+        C = np.eye(n - 1) + Xt @ Xt.T / lam
+        res = minimize_scalar(lambda ls2: -multivariate_normal(mean=np.zeros(n - 1), cov=np.exp(ls2) * C).logpdf(yt),
+                              bounds=(-20, 20), method="bounded", options={"xatol": 1e-10})
+        assert -res.fun == pytest.approx(l_val + const, abs=1e-6)
+
+
+def test_ridge_evidence_residual_identity_and_limits():
+    r = np.random.default_rng(32)
+    n, d = 300, 16
+    X = r.standard_normal((n, d))
+    X /= np.linalg.norm(X, axis=1, keepdims=True)
+    y = X @ r.standard_normal(d) + 0.2 * r.standard_normal(n)
+    grid = O.lambda_grid()
+    L = O.ridge_log_evidence(X, y, grid)
+    # r(lam) = |y_c - X_c a|^2 + lam |a|^2 at the ridge solution (solved by a different routine)
+    Xc, yc = X - X.mean(axis=0), y - y.mean()
+    theta = np.linalg.eigvalsh(Xc.T @ Xc)
+    for lam, l_val in zip(grid[::6], L[::6]):
+        a, _ = O.ridge_fit(X, y, lam)
+        rr = np.sum((yc - Xc @ a) ** 2) + lam * (a @ a)
+        assert l_val == pytest.approx(-0.5 * (n - 1) * np.log(rr) - 0.5 * np.log1p(theta / lam).sum(), rel=1e-9)
+    # a noiseless linear target wants the weakest penalty, pure noise the strongest
+    assert O.select_lambda(X, X @ r.standard_normal(d) * 5.0, grid) == 0
+    assert O.select_lambda(X, r.standard_normal(n), grid) == len(grid) - 1
+    # fewer than two pairs: nothing to judge by
+    assert O.select_lambda(X[:1], y[:1], grid) == len(grid) // 2
+    assert O.select_lambda(X[:1], y[:1], grid, default_index=3) == 3
+
+
+def test_ridge_evidence_recovers_a_planted_prior_precision():
+    """Data drawn from the model itself (a ~ N(0, s2/lam I), noise s2): the selected penalty lands next to lam."""
+    r = np.random.default_rng(33)
+    n, d, s2 = 4000, 48, 0.25
+    grid = O.lambda_grid()
+    for lam_true in (0.1, 3.0):
+        X = r.standard_normal((n, d))
+        a = r.standard_normal(d) * np.sqrt(s2 / lam_true)
+        y = X @ a + np.sqrt(s2) * r.standard_normal(n) + 1.0
+        lam_sel = grid[O.select_lambda(X, y, grid)]
+        assert abs(np.log10(lam_sel / lam_true)) <= 0.5, (lam_true, lam_sel)
+
+
 def test_fit_predictor_against_brute_force_removal_costs():
     """Fit on routed calibration pairs; exp(s-hat) is unbiased on them and beats the static score
     out of sample when the energy depends on the token's direction."""
