@@ -277,6 +277,8 @@ int base_exact_removal_error(const base_layer_shape* shape, const base_layer_wei
  *   base_calib_reset(state)
  *   for every batch:  base_calib_accumulate(batch, state)             -- pass 1: statistics
  *   base_calib_solve(state, lambda)                                   -- a_u = (G_c + lambda I)^-1 q_c, b_u
+ *     or: base_calib_select_lambda(state, grid) then base_calib_solve_selected(state)
+ *                                                                     -- lambda per expert by marginal likelihood
  *   for every batch:  base_calib_accumulate_correction(batch, state)  -- pass 2: sum of exp(s-hat)
  *   base_calib_finalize(state, pred_A, pred_b)                        -- b_u += log(mean energy / mean exp(s-hat))
  *
@@ -293,9 +295,25 @@ int base_exact_removal_error(const base_layer_shape* shape, const base_layer_wei
  * pred_A, fp32 pred_b). weights->pred_A / pred_b must point to valid buffers during calibration
  * (their values do not matter: without a budget the selection has no effect).
  *
+ * select_lambda evaluates, for every expert independently, the log marginal likelihood of each of the
+ * n_lambda candidate penalties (a HOST array of 1..32 positive values; the paper uses 25 values
+ * logarithmically spaced from 1e-4 to 1e2) under the model behind the centred ridge -- coefficients
+ * N(0, s2/lambda I), flat prior on the intercept, noise variance s2 at its maximising value:
+ *     L(lambda) = -(n-1)/2 log r(lambda) - 1/2 (log det(G_c + lambda I) - d log lambda),
+ *     r(lambda) = y_c.y_c - q_c^T (G_c + lambda I)^-1 q_c, floored at 1e-12 y_c.y_c + 1e-300
+ * (the paper names the criterion without a formula; it evaluates all penalties from one
+ * eigendecomposition per expert, here each penalty takes one fp64 Cholesky factorisation, which yields
+ * the same two quantities). The candidate of largest L (the first on a tie) becomes the expert's lambda;
+ * a candidate for which the stored (fp32) Gram matrix makes G_c + lambda I indefinite gets L = -inf; an
+ * expert with fewer than two pairs takes candidate n_lambda/2. solve_selected then solves every expert
+ * with its own lambda. Its `workspace`: base_calib_select_workspace_bytes(shape) = E*d*d*8 bytes,
+ * 256-byte aligned.
+ *
  * `state` is a caller-owned device buffer of base_calib_state_bytes(shape) bytes, 256-byte aligned,
  * holding in this order (each array 256-byte aligned): n, sum_y, sum_yy, sum_e, sum_p, coef_b
- * ([E] fp64 each); sum_z, sum_yz, coef_a ([E,d] fp64 each); gram ([E,d,d] fp32); cg_iters ([E] int32).
+ * ([E] fp64 each); sum_z, sum_yz, coef_a ([E,d] fp64 each); gram ([E,d,d] fp32); cg_iters ([E] int32);
+ * lambda ([E] fp64, the selected penalties); evidence ([E,32] fp64, L of every candidate); lambda_index
+ * ([E] int32).
  * `workspace`: base_calib_workspace_bytes(shape, T_max) bytes, 1024-byte aligned. Limits: those of the
  * layer, and d a multiple of 128, d <= 4096. Errors as for base_moe_decode_layer; 0 bytes = unsupported.
  */
@@ -306,6 +324,10 @@ int base_calib_accumulate(const base_layer_shape* shape, const base_layer_weight
                           const float* router_logits, int T, void* state, size_t state_bytes, void* workspace,
                           size_t workspace_bytes, void* stream);
 int base_calib_solve(const base_layer_shape* shape, void* state, size_t state_bytes, double lambda, void* stream);
+size_t base_calib_select_workspace_bytes(const base_layer_shape* shape);
+int base_calib_select_lambda(const base_layer_shape* shape, void* state, size_t state_bytes, const double* h_lambdas,
+                             int n_lambda, void* workspace, size_t workspace_bytes, void* stream);
+int base_calib_solve_selected(const base_layer_shape* shape, void* state, size_t state_bytes, void* stream);
 int base_calib_accumulate_correction(const base_layer_shape* shape, const base_layer_weights* weights,
                                      const void* hidden_bf16, const float* router_logits, int T, void* state,
                                      size_t state_bytes, void* workspace, size_t workspace_bytes, void* stream);

@@ -31,6 +31,7 @@ EXPORTS = (
     "base_last_launch_count", "base_true_removal_costs", "base_energy_retained", "base_exact_removal_error",
     "base_calib_state_bytes", "base_calib_workspace_bytes", "base_calib_reset", "base_calib_accumulate",
     "base_calib_solve", "base_calib_accumulate_correction", "base_calib_finalize",
+    "base_calib_select_workspace_bytes", "base_calib_select_lambda", "base_calib_solve_selected",
     "base_status_string", "base_last_cuda_error",
 )
 
@@ -102,6 +103,11 @@ def lib():
     L.base_calib_accumulate.argtypes = batch_args
     L.base_calib_accumulate_correction.argtypes = batch_args
     L.base_calib_solve.argtypes = [C.POINTER(LayerShape), vp, C.c_size_t, C.c_double, vp]
+    L.base_calib_select_workspace_bytes.argtypes = [C.POINTER(LayerShape)]
+    L.base_calib_select_workspace_bytes.restype = C.c_size_t
+    L.base_calib_select_lambda.argtypes = [C.POINTER(LayerShape), vp, C.c_size_t, C.POINTER(C.c_double), ip, vp,
+                                           C.c_size_t, vp]
+    L.base_calib_solve_selected.argtypes = [C.POINTER(LayerShape), vp, C.c_size_t, vp]
     L.base_calib_finalize.argtypes = [C.POINTER(LayerShape), vp, C.c_size_t, vp, vp, vp]
     L.base_profile_events.argtypes = [C.POINTER(C.c_void_p)]
     L.base_last_launch_count.restype = ip
@@ -353,6 +359,23 @@ class Calibrator:
     def solve(self, lam, stream=None):
         _check(lib().base_calib_solve(C.byref(self._s), _ptr(self.state), self.state.numel(), float(lam), _stream(stream)))
 
+    def select_lambda(self, lambdas=None, stream=None):
+        """Ridge penalty per expert by marginal likelihood over `lambdas` (default: the paper's grid, 25 values
+        logarithmically spaced from 1e-4 to 1e2); returns the grid. Follow with solve_selected()."""
+        if lambdas is None:
+            lambdas = [1e-4 * (1e6 ** (i / 24.0)) for i in range(25)]
+        lambdas = [float(v) for v in lambdas]
+        n_ws = lib().base_calib_select_workspace_bytes(C.byref(self._s))
+        if getattr(self, "_select_ws", None) is None or self._select_ws.numel() < n_ws:
+            self._select_ws = alloc_workspace(n_ws, self.state.device)
+        arr = (C.c_double * len(lambdas))(*lambdas)
+        _check(lib().base_calib_select_lambda(C.byref(self._s), _ptr(self.state), self.state.numel(), arr, len(lambdas),
+                                              _ptr(self._select_ws), self._select_ws.numel(), _stream(stream)))
+        return lambdas
+
+    def solve_selected(self, stream=None):
+        _check(lib().base_calib_solve_selected(C.byref(self._s), _ptr(self.state), self.state.numel(), _stream(stream)))
+
     def accumulate_correction(self, weights, hidden, router_logits=None, stream=None):
         self._batch(lib().base_calib_accumulate_correction, weights, hidden, router_logits, stream)
 
@@ -383,6 +406,10 @@ class Calibrator:
         take("gram", E * d * d, torch.float32, 4)
         out["gram"] = out["gram"].view(E, d, d)
         take("cg_iters", E, torch.int32, 4)
+        take("lambda", E, torch.float64, 8)
+        take("evidence", E * 32, torch.float64, 8)
+        out["evidence"] = out["evidence"].view(E, 32)
+        take("lambda_index", E, torch.int32, 4)
         return out
 
 

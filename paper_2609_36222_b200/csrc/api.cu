@@ -417,6 +417,32 @@ int base_calib_solve(const base_layer_shape* shape, void* state, size_t state_by
   return e == cudaSuccess ? BASE_OK : cuda_fail(e);
 }
 
+size_t base_calib_select_workspace_bytes(const base_layer_shape* shape) {
+  if (check_shape(shape, 1) != BASE_OK || shape->d % 128 != 0 || shape->d > 4096) return 0;
+  return calib_evidence_scratch_bytes(*shape);
+}
+
+int base_calib_select_lambda(const base_layer_shape* shape, void* state, size_t state_bytes, const double* h_lambdas,
+                             int n_lambda, void* workspace, size_t workspace_bytes, void* stream) {
+  int rc = check_calib(shape, state, state_bytes);
+  if (rc != BASE_OK) return rc;
+  if (!h_lambdas || n_lambda < 1 || n_lambda > kCalibMaxLambdas) return BASE_ERR_INVALID_ARG;
+  for (int i = 0; i < n_lambda; ++i)
+    if (!(h_lambdas[i] > 0.0)) return BASE_ERR_INVALID_ARG;
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return BASE_ERR_INVALID_ARG;
+  if (calib_evidence_scratch_bytes(*shape) > workspace_bytes) return BASE_ERR_WORKSPACE_TOO_SMALL;
+  cudaError_t e = launch_calib_evidence(*shape, carve_calib_state(state, *shape), workspace, h_lambdas, n_lambda,
+                                        n_lambda / 2, static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? BASE_OK : cuda_fail(e);
+}
+
+int base_calib_solve_selected(const base_layer_shape* shape, void* state, size_t state_bytes, void* stream) {
+  int rc = check_calib(shape, state, state_bytes);
+  if (rc != BASE_OK) return rc;
+  cudaError_t e = launch_calib_solve(*shape, carve_calib_state(state, *shape), 0.0, static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? BASE_OK : cuda_fail(e);
+}
+
 int base_calib_accumulate_correction(const base_layer_shape* shape, const base_layer_weights* weights,
                                      const void* hidden_bf16, const float* router_logits, int T, void* state,
                                      size_t state_bytes, void* workspace, size_t workspace_bytes, void* stream) {

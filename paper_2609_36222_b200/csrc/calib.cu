@@ -239,3 +239,4 @@ __global__ void __launch_bounds__(256) calib_vector_reduce_kernel(const int32_t*
 
 #include "calib_gram.cuh"
 #include "calib_solve.cuh"
+#include "calib_evidence.cuh"

@@ -4,6 +4,8 @@
 
 namespace base {
 
+constexpr int kCalibMaxLambdas = 32;   // candidate ridge penalties per selection (the paper's grid has 25)
+
 // Sufficient statistics of one layer, per expert. Vector and scalar statistics are fp64, the Gram
 // matrices fp32. The fitted coefficients live in the same buffer so that the correction pass and
 // the final rounding can find them.
@@ -19,6 +21,9 @@ struct CalibState {
   double* coef_a;   // [E,d] fitted coefficients
   float* gram;      // [E,d,d] sum of zbar zbar^T
   int32_t* iters;   // [E] conjugate-gradient iterations of the last solve (diagnostic)
+  double* lambda;   // [E] ridge penalty chosen by the evidence (0 until a selection has run)
+  double* evidence; // [E, kCalibMaxLambdas] log marginal likelihood of every candidate of the last selection
+  int32_t* lambda_index;   // [E] index of the chosen candidate
   size_t bytes;
 };
 
@@ -44,6 +49,9 @@ inline CalibState carve_calib_state(void* base_ptr, const base_layer_shape& s) {
   c.coef_a = static_cast<double*>(take(E * d * 8));
   c.gram = static_cast<float*>(take(E * d * d * 4));
   c.iters = static_cast<int32_t*>(take(E * 4));
+  c.lambda = static_cast<double*>(take(E * 8));
+  c.evidence = static_cast<double*>(take(E * kCalibMaxLambdas * 8));
+  c.lambda_index = static_cast<int32_t*>(take(E * 4));
   c.bytes = align_up(off, 1024);
   return c;
 }
@@ -88,7 +96,13 @@ inline CalibScratch carve_calib_scratch(void* base_ptr, const base_layer_shape& 
 cudaError_t launch_calib_accumulate(const base_layer_shape& s, const Workspace& ws, const CalibScratch& sc,
                                     const CalibState& st, const void* hidden, int n_split, int T, cudaStream_t stream,
                                     int* launches);
-// Centred ridge solve per expert (conjugate gradients on the fp32 Gram matrix, fp64 vectors).
+// Evidence of every candidate penalty per expert (one Cholesky factorisation each) and the best one into
+// st.lambda; scratch: calib_evidence_scratch_bytes(s) bytes. lambdas is a HOST array.
+size_t calib_evidence_scratch_bytes(const base_layer_shape& s);
+cudaError_t launch_calib_evidence(const base_layer_shape& s, const CalibState& st, void* scratch, const double* lambdas,
+                                  int n_lambda, int default_index, cudaStream_t stream);
+// Centred ridge solve per expert (conjugate gradients on the fp32 Gram matrix, fp64 vectors);
+// lambda <= 0: every expert uses its own st.lambda.
 cudaError_t launch_calib_solve(const base_layer_shape& s, const CalibState& st, double lambda, cudaStream_t stream);
 // Correction pass: adds sum exp(s-hat) of the routed pairs of this batch (routes must be in the workspace).
 cudaError_t launch_calib_correction(const base_layer_shape& s, const Workspace& ws, const CalibScratch& sc,

@@ -1,0 +1,240 @@
+// Ridge penalty per expert by marginal likelihood (App. Calibration Details): for every candidate
+// lambda the evidence of the centred ridge model needs log det(G_c + lambda I) and the quadratic form
+// q_c^T (G_c + lambda I)^-1 q_c. Both come out of one Cholesky factorisation G_c + lambda I = L L^T:
+// log det = 2 sum log L_ii, and with w = L^-1 q_c the quadratic form is |w|^2. (The paper takes one
+// eigendecomposition per expert and evaluates all penalties from it; a factorisation per penalty gives
+// the same numbers, is exact for repeated and zero eigenvalues, and needs no eigen-solver on the
+// device.) One CTA per expert, fp64 throughout, the matrix in a global scratch square of d x d
+// doubles per expert. Included by calib.cu.
+#pragma once
+
+namespace base {
+
+namespace {
+
+constexpr int kEvThreads = 256;
+constexpr int kEvNb = 32;      // panel width
+constexpr int kEvTile = 64;    // trailing-update tile
+
+struct LambdaGrid {
+  double v[kCalibMaxLambdas];
+  int n;
+  int default_index;   // for experts with fewer than two pairs
+};
+
+// Cholesky of the 32 x 32 diagonal block held in shared memory (row stride 33), by one warp; lane = row.
+// Returns the sum of log L_jj over the block through *logsum (lane 0) and clears *ok on a pivot <= 0.
+__device__ __forceinline__ void ev_factor_diag(double (*D)[kEvNb + 1], int lane, double* logsum, int* ok) {
+  double ls = 0.0;
+  for (int j = 0; j < kEvNb; ++j) {
+    double djj = D[j][j];
+    if (!(djj > 0.0)) {
+      if (lane == 0) *ok = 0;
+      djj = 1.0;
+    }
+    djj = sqrt(djj);
+    ls += log(djj);
+    __syncwarp();
+    double lij = 0.0;
+    if (lane == j) D[j][j] = djj;
+    if (lane > j) {
+      lij = D[lane][j] / djj;
+      D[lane][j] = lij;
+    }
+    __syncwarp();
+    if (lane > j)
+      for (int c = j + 1; c <= lane; ++c) D[lane][c] -= lij * D[c][j];
+    __syncwarp();
+  }
+  if (lane == 0) *logsum += ls;
+}
+
+__global__ void __launch_bounds__(kEvThreads) calib_evidence_kernel(CalibState st, double* __restrict__ chol, int d,
+                                                                    LambdaGrid grid) {
+  extern __shared__ double s_ev[];
+  double* m = s_ev;                 // [d] mean of the inputs
+  double* qc = m + d;               // [d] centred cross-moment
+  double* w = qc + d;               // [d] running right-hand side of the forward solve
+  double* At = w + d;               // [kEvNb][kEvTile] panel rows of the tile's row block, transposed
+  double* Bt = At + kEvNb * kEvTile;   // ... of its column block
+  __shared__ double D[kEvNb][kEvNb + 1];
+  __shared__ double s_logsum;
+  __shared__ int s_pd;
+  const int u = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const double n = st.n[u];
+  double* ev_out = st.evidence + size_t(u) * kCalibMaxLambdas;
+  if (n < 2.0) {
+    if (tid == 0) {
+      st.lambda_index[u] = grid.default_index;
+      st.lambda[u] = grid.v[grid.default_index];
+    }
+    for (int i = tid; i < kCalibMaxLambdas; i += kEvThreads) ev_out[i] = 0.0;
+    return;
+  }
+  const double sy = st.sum_y[u];
+  for (int j = tid; j < d; j += kEvThreads) {
+    const double mj = st.sum_z[size_t(u) * d + j] / n;
+    m[j] = mj;
+    qc[j] = st.sum_yz[size_t(u) * d + j] - sy * mj;
+  }
+  __syncthreads();
+  const double yy = st.sum_yy[u] - sy * sy / n;
+  const double r_floor = 1e-12 * yy + 1e-300;
+  const float* G = st.gram + size_t(u) * d * d;
+  double* A = chol + size_t(u) * d * d;
+  double best = 0.0;
+  int best_i = -1;
+
+  for (int li = 0; li < grid.n; ++li) {
+    const double lam = grid.v[li];
+    // ---- A (lower triangle) = G - n m m^T + lambda I
+    for (int i = warp; i < d; i += kEvThreads / 32) {
+      const double nmi = n * m[i];
+      for (int j = lane; j <= i; j += 32)
+        A[size_t(i) * d + j] = double(G[size_t(i) * d + j]) - nmi * m[j] + (i == j ? lam : 0.0);
+    }
+    for (int j = tid; j < d; j += kEvThreads) w[j] = qc[j];
+    if (tid == 0) {
+      s_logsum = 0.0;
+      s_pd = 1;
+    }
+    __syncthreads();
+    double wnorm2 = 0.0;   // accumulated by warp 0 / lane 0 only
+
+    for (int k0 = 0; k0 < d; k0 += kEvNb) {
+      // ---- diagonal block: factor, then the block's part of w = L^-1 q
+      for (int idx = tid; idx < kEvNb * kEvNb; idx += kEvThreads) {
+        const int i = idx >> 5, j = idx & 31;
+        D[i][j] = j <= i ? A[size_t(k0 + i) * d + k0 + j] : 0.0;
+      }
+      __syncthreads();
+      if (warp == 0) {
+        ev_factor_diag(D, lane, &s_logsum, &s_pd);
+        for (int j = 0; j < kEvNb; ++j) {
+          const double wj = w[k0 + j] / D[j][j];
+          __syncwarp();
+          if (lane == j) w[k0 + j] = wj;
+          if (lane > j) w[k0 + lane] -= D[lane][j] * wj;
+          __syncwarp();
+        }
+        const double wl = w[k0 + lane];
+        double s2 = wl * wl;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) s2 += __shfl_down_sync(0xffffffffu, s2, o);
+        wnorm2 += s2;
+      }
+      __syncthreads();
+      const int r0 = k0 + kEvNb;
+      const int mrows = d - r0;
+      if (mrows <= 0) break;
+      // ---- panel: X = A21 L11^-T, row by row (one thread per row), and w_rest -= X w_k
+      for (int i = r0 + tid; i < d; i += kEvThreads) {
+        double x[kEvNb];
+        double* row = A + size_t(i) * d + k0;
+#pragma unroll
+        for (int j = 0; j < kEvNb; ++j) x[j] = row[j];
+        double dot = 0.0;
+#pragma unroll
+        for (int j = 0; j < kEvNb; ++j) {
+          double v = x[j];
+#pragma unroll
+          for (int c = 0; c < j; ++c) v -= x[c] * D[j][c];
+          v /= D[j][j];
+          x[j] = v;
+          dot += v * w[k0 + j];
+        }
+#pragma unroll
+        for (int j = 0; j < kEvNb; ++j) row[j] = x[j];
+        w[i] -= dot;
+      }
+      __syncthreads();
+      // ---- trailing update of the lower triangle: C -= X_bi X_bj^T in 64 x 64 tiles
+      const int mt = (mrows + kEvTile - 1) / kEvTile;
+      const int ty = tid >> 4, tx = tid & 15;
+      for (int bi = 0; bi < mt; ++bi) {
+        for (int bj = 0; bj <= bi; ++bj) {
+          // stage the two row blocks of the panel, transposed: At[k][row], Bt[k][row]
+          {
+            const int i = tid & 63, kg = tid >> 6;   // 64 rows x 4 groups of 8 columns
+            const int ga = r0 + bi * kEvTile + i, gb = r0 + bj * kEvTile + i;
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+              const int kk = kg * 8 + k;
+              At[kk * kEvTile + i] = ga < d ? A[size_t(ga) * d + k0 + kk] : 0.0;
+              Bt[kk * kEvTile + i] = gb < d ? A[size_t(gb) * d + k0 + kk] : 0.0;
+            }
+          }
+          __syncthreads();
+          double acc[4][4] = {};
+#pragma unroll 8
+          for (int k = 0; k < kEvNb; ++k) {
+            const double2 a01 = *reinterpret_cast<const double2*>(At + k * kEvTile + ty * 4);
+            const double2 a23 = *reinterpret_cast<const double2*>(At + k * kEvTile + ty * 4 + 2);
+            const double2 b01 = *reinterpret_cast<const double2*>(Bt + k * kEvTile + tx * 4);
+            const double2 b23 = *reinterpret_cast<const double2*>(Bt + k * kEvTile + tx * 4 + 2);
+            const double a[4] = {a01.x, a01.y, a23.x, a23.y}, b[4] = {b01.x, b01.y, b23.x, b23.y};
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+              for (int j = 0; j < 4; ++j) acc[i][j] = fma(a[i], b[j], acc[i][j]);
+          }
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const int gi = r0 + bi * kEvTile + ty * 4 + i;
+            if (gi >= d) continue;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const int gj = r0 + bj * kEvTile + tx * 4 + j;
+              if (gj <= gi) A[size_t(gi) * d + gj] -= acc[i][j];
+            }
+          }
+          __syncthreads();
+        }
+      }
+    }
+    // ---- evidence of this penalty
+    if (tid == 0) {
+      double ev;
+      if (s_pd) {
+        const double r = fmax(yy - wnorm2, r_floor);
+        ev = -0.5 * (n - 1.0) * log(r) - 0.5 * (2.0 * s_logsum - double(d) * log(lam));
+      } else {
+        ev = -INFINITY;   // rounding of the stored Gram matrix made G_c + lambda I indefinite: not a candidate
+      }
+      ev_out[li] = ev;
+      if (best_i < 0 || ev > best) {
+        best = ev;
+        best_i = li;
+      }
+    }
+    __syncthreads();
+  }
+  if (tid == 0) {
+    for (int i = grid.n; i < kCalibMaxLambdas; ++i) ev_out[i] = 0.0;
+    st.lambda_index[u] = best_i;
+    st.lambda[u] = grid.v[best_i];
+  }
+}
+
+}  // namespace
+
+size_t calib_evidence_scratch_bytes(const base_layer_shape& s) { return size_t(s.E) * s.d * s.d * sizeof(double); }
+
+cudaError_t launch_calib_evidence(const base_layer_shape& s, const CalibState& st, void* scratch, const double* lambdas,
+                                  int n_lambda, int default_index, cudaStream_t stream) {
+  LambdaGrid g{};
+  g.n = n_lambda;
+  g.default_index = default_index;
+  for (int i = 0; i < n_lambda; ++i) g.v[i] = lambdas[i];
+  const size_t smem = (size_t(3) * s.d + 2 * kEvNb * kEvTile) * sizeof(double);
+  static size_t set_for = 0;
+  if (smem > set_for) {
+    cudaError_t a = cudaFuncSetAttribute(calib_evidence_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+    if (a != cudaSuccess) return a;
+    set_for = smem;
+  }
+  calib_evidence_kernel<<<s.E, kEvThreads, smem, stream>>>(st, static_cast<double*>(scratch), s.d, g);
+  return cudaGetLastError();
+}
+
+}  // namespace base

@@ -24,8 +24,9 @@ __device__ __forceinline__ double block_sum(double v, double* s_red) {
 // a = (G_c + lambda I)^-1 q_c and b = ybar - a . zbar_mean for one expert per CTA (Eq. of App.
 // Calibration Details), by conjugate gradients: G_c v = G v - n m (m . v) is applied without forming
 // the centred matrix. Vectors are fp64 in shared memory, the Gram matrix is read as stored (fp32).
-__global__ void __launch_bounds__(kSolveThreads) calib_solve_kernel(CalibState st, int d, double lambda, int iter_cap) {
+__global__ void __launch_bounds__(kSolveThreads) calib_solve_kernel(CalibState st, int d, double lambda_all, int iter_cap) {
   extern __shared__ double s_vec[];
+  const double lambda = lambda_all > 0.0 ? lambda_all : st.lambda[blockIdx.x];   // one penalty for all, or the expert's own
   double* m = s_vec;          // mean of the inputs
   double* x = m + d;          // solution
   double* r = x + d;          // residual

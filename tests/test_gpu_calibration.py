@@ -135,6 +135,126 @@ def test_calibration_end_to_end_matches_oracle_fit():
     assert 1 - ((y - s_dev) ** 2).sum() / ((y - y.mean()) ** 2).sum() > 0.5
 
 
+def _evidence_from_statistics(st, u, d, lambdas):
+    """fp64 NumPy evidence of expert u from the device's own statistics (the matrix the kernel factors: lower
+    triangle of the stored Gram matrix, centred), by Cholesky; None where that matrix is not positive definite."""
+    n = float(st["n"][u])
+    m = st["sum_z"][u] / n
+    G = st["gram"][u].astype(np.float64)
+    G = np.tril(G) + np.tril(G, -1).T
+    Gc = G - n * np.outer(m, m)
+    qc = st["sum_yz"][u] - st["sum_y"][u] * m
+    yy = st["sum_yy"][u] - st["sum_y"][u] ** 2 / n
+    out = []
+    for lam in lambdas:
+        try:
+            L = np.linalg.cholesky(Gc + lam * np.eye(d))
+        except np.linalg.LinAlgError:
+            out.append(None)
+            continue
+        w = np.linalg.solve(L, qc)
+        r = max(yy - w @ w, 1e-12 * yy + 1e-300)
+        out.append(-0.5 * (n - 1) * np.log(r) - 0.5 * (2 * np.log(np.diag(L)).sum() - d * np.log(lam)))
+    return out
+
+
+@pytest.mark.parametrize("name,sizes,alpha", [("tiny", (96, 128, 50, 110), 0.5), ("mid", (256, 200), None)])
+def test_lambda_by_evidence_matches_numpy_on_the_device_statistics(name, sizes, alpha):
+    cfg = wl.CONFIGS[name]
+    kw = {} if alpha is None else {"planted_alpha": alpha}
+    base, batches = _batches(cfg, sizes, **kw)
+    dl = device_layer_from_host(base, DEV, T_max=max(sizes))
+    cal = B.Calibrator(dl.shape, max(sizes), DEV)
+    for h in batches:
+        lg = O.router_logits(h.z, base.router_w, base.router_bias)
+        cal.accumulate(dl.weights, bits_to_device(h.hidden_bits, DEV), router_logits=torch.from_numpy(lg).to(DEV))
+    grid = cal.select_lambda()
+    np.testing.assert_allclose(grid, O.lambda_grid(), rtol=1e-12)
+    torch.cuda.synchronize()
+    st = {k: v.cpu().numpy() for k, v in cal.statistics().items()}
+    d, E = cfg.d, cfg.E
+    order = np.argsort(-st["n"])
+    fitted = [u for u in order if st["n"][u] >= 2]
+    # every expert on the small shape; the most, a middling and the least used one on the large shape
+    check = fitted if d <= 512 else [fitted[0], fitted[len(fitted) // 2], fitted[-1]]
+    which = range(len(grid)) if d <= 512 else range(0, len(grid), 4)
+    for u in check:
+        ref = _evidence_from_statistics(st, u, d, [grid[i] for i in which])
+        for i, r in zip(which, ref):
+            ev = st["evidence"][u, i]
+            if r is None:
+                assert ev == -np.inf or ev < -1e300
+            else:
+                assert abs(ev - r) <= 1e-7 * (abs(r) + st["n"][u] + d), (u, i, ev, r)
+    for u in range(E):
+        ev = st["evidence"][u, :len(grid)]
+        if st["n"][u] < 2:
+            assert st["lambda_index"][u] == len(grid) // 2
+        else:
+            assert st["lambda_index"][u] == int(np.argmax(ev))            # first maximum
+        assert st["lambda"][u] == grid[st["lambda_index"][u]]
+    # the solve with the selected penalties: predictions on the expert's statistics against NumPy
+    cal.solve_selected()
+    torch.cuda.synchronize()
+    st2 = {k: v.cpu().numpy() for k, v in cal.statistics().items() if k != "gram"}
+    for u in check[:3]:
+        n = float(st["n"][u])
+        m = st["sum_z"][u] / n
+        G = st["gram"][u].astype(np.float64)
+        Gc = 0.5 * (G + G.T) - n * np.outer(m, m)
+        qc = st["sum_yz"][u] - st["sum_y"][u] * m
+        a_ref = np.linalg.solve(Gc + st["lambda"][u] * np.eye(d), qc)
+        # compare through the quantity the fit minimises: a difference in a weighs by the Gram matrix
+        da = st2["coef_a"][u] - a_ref
+        assert da @ (Gc @ da) + st["lambda"][u] * (da @ da) <= 1e-10 * max(qc @ a_ref, 1e-30)
+
+
+def test_lambda_by_evidence_end_to_end_against_the_oracle():
+    """Selected penalties and deployed coefficients against the oracle's fit with the same grid (its energies
+    come from fp64 experts, the device's carry the FFN's error, so near-ties may fall one grid step apart)."""
+    cfg = wl.CONFIGS["tiny"]
+    sizes = (128, 128, 128, 128)
+    base, batches = _batches(cfg, sizes, planted_alpha=0.5)
+    dl = device_layer_from_host(base, DEV, T_max=max(sizes))
+    cal = B.Calibrator(dl.shape, max(sizes), DEV)
+    logits = []
+    for h in batches:
+        lg = O.router_logits(h.z, base.router_w, base.router_bias)
+        logits.append(lg)
+        cal.accumulate(dl.weights, bits_to_device(h.hidden_bits, DEV), router_logits=torch.from_numpy(lg).to(DEV))
+    grid = np.array(cal.select_lambda())
+    cal.solve_selected()
+    for h, lg in zip(batches, logits):
+        cal.accumulate_correction(dl.weights, bits_to_device(h.hidden_bits, DEV), router_logits=torch.from_numpy(lg).to(DEV))
+    A_dev, b_dev = cal.finalize()
+    torch.cuda.synchronize()
+    A_dev, b_dev = A_dev.float().cpu().numpy().astype(np.float64), b_dev.cpu().numpy().astype(np.float64)
+    idx_dev = cal.statistics()["lambda_index"].cpu().numpy()
+    z = np.concatenate([h.z for h in batches])
+    lg = np.concatenate(logits)
+    zbar = O.normalise(z)
+    _, R, _, _, _ = O.route_topk(lg, cfg.K)
+    A_ref, b_ref = O.fit_predictor(z, lg, base.expert_weights, cfg.K, cfg.E, lam=grid, eps=EPS)
+    same, worst = 0, 0.0
+    for u in range(cfg.E):
+        tt = np.nonzero((R == u).any(axis=1))[0]
+        if tt.size < 2:
+            continue
+        out = O.expert_ffn(z[tt], *base.expert_weights(u))
+        y = np.log((out * out).sum(axis=1) + EPS)
+        L_ref = O.ridge_log_evidence(zbar[tt], y, grid)
+        i_ref = int(np.argmax(L_ref))
+        # the evidence is flat around its maximum: the device's choice must be a neighbour of the oracle's and
+        # as good as it within a Bayes factor of e^0.5
+        assert abs(int(idx_dev[u]) - i_ref) <= 1, (u, idx_dev[u], i_ref)
+        assert L_ref[i_ref] - L_ref[int(idx_dev[u])] <= 0.5, (u, L_ref[i_ref] - L_ref[int(idx_dev[u])])
+        same += int(idx_dev[u]) == i_ref
+        if int(idx_dev[u]) == i_ref:
+            worst = max(worst, np.abs(zbar[tt] @ (A_dev[u] - A_ref[u]) + b_dev[u] - b_ref[u]).max())
+    assert same >= 0.5 * cfg.E
+    assert worst <= 5e-2, worst
+
+
 def test_calibration_error_codes():
     cfg = wl.CONFIGS["tiny"]
     with pytest.raises(B.BaseError, match="unsupported"):
@@ -142,6 +262,10 @@ def test_calibration_error_codes():
     cal = B.Calibrator((cfg.d, cfg.E, cfg.K, cfg.I), 8, DEV)
     with pytest.raises(B.BaseError, match="invalid"):
         cal.solve(0.0)
+    with pytest.raises(B.BaseError, match="invalid"):
+        cal.select_lambda([1e-2, -1.0])
+    with pytest.raises(B.BaseError, match="invalid"):
+        cal.select_lambda([1.0] * 33)
 
 
 def test_device_fitted_predictor_drives_the_layer():
