@@ -12,7 +12,7 @@ namespace base {
 
 namespace {
 
-constexpr int kEvThreads = 256;
+constexpr int kEvThreads = 512;
 constexpr int kEvNb = 32;      // panel width
 constexpr int kEvTile = 64;    // trailing-update tile
 
@@ -56,7 +56,7 @@ __global__ void __launch_bounds__(kEvThreads) calib_evidence_kernel(CalibState s
   double* qc = m + d;               // [d] centred cross-moment
   double* w = qc + d;               // [d] running right-hand side of the forward solve
   double* At = w + d;               // [kEvNb][kEvTile] panel rows of the tile's row block, transposed
-  double* Bt = At + kEvNb * kEvTile;   // ... of its column block
+  double* Bt = At + kEvNb * kEvTile;   // [kEvNb][2 * kEvTile] ... of its column block (128 columns)
   __shared__ double D[kEvNb][kEvNb + 1];
   __shared__ double s_logsum;
   __shared__ int s_pd;
@@ -148,20 +148,42 @@ __global__ void __launch_bounds__(kEvThreads) calib_evidence_kernel(CalibState s
         w[i] -= dot;
       }
       __syncthreads();
-      // ---- trailing update of the lower triangle: C -= X_bi X_bj^T in 64 x 64 tiles
+      // ---- trailing update of the lower triangle: C -= X_bi X_bj^T in tiles of 64 rows x 128 columns
       const int mt = (mrows + kEvTile - 1) / kEvTile;
-      const int ty = tid >> 4, tx = tid & 15;
+      // a warp owns 4 rows of the tile, a lane the columns {2 tx, 2 tx + 1} and {64 + 2 tx, 64 + 2 tx + 1}
+      const int ty = tid >> 5, tx = tid & 31;
       for (int bi = 0; bi < mt; ++bi) {
-        for (int bj = 0; bj <= bi; ++bj) {
-          // stage the two row blocks of the panel, transposed: At[k][row], Bt[k][row]
+        // the row block of the panel is staged once per tile row, transposed: At[k][row]
+        {
+          const int i = tid & 63, kg = tid >> 6;   // 64 rows x 8 groups of 4 columns
+          const int ga = r0 + bi * kEvTile + i;
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            const int kk = kg * 4 + k;
+            At[kk * kEvTile + i] = ga < d ? A[size_t(ga) * d + k0 + kk] : 0.0;
+          }
+        }
+        for (int bj = 0; bj * 2 <= bi; ++bj) {
+          const int c0 = r0 + bj * 2 * kEvTile;
+          // the tile of C is requested first, so that its latency hides behind the staging and the products
+          double cval[4][4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const int gi = r0 + bi * kEvTile + ty * 4 + i;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const int gj = c0 + (j >> 1) * kEvTile + tx * 2 + (j & 1);
+              cval[i][j] = (gi < d && gj <= gi) ? A[size_t(gi) * d + gj] : 0.0;
+            }
+          }
           {
-            const int i = tid & 63, kg = tid >> 6;   // 64 rows x 4 groups of 8 columns
-            const int ga = r0 + bi * kEvTile + i, gb = r0 + bj * kEvTile + i;
+            const int i = tid & 127, kg = tid >> 7;   // 128 rows x 4 groups of 8 columns
+            const int gb = c0 + i;
+            const bool in = gb < d && gb <= r0 + bi * kEvTile + kEvTile - 1;   // rows past the diagonal block are not needed
 #pragma unroll
             for (int k = 0; k < 8; ++k) {
               const int kk = kg * 8 + k;
-              At[kk * kEvTile + i] = ga < d ? A[size_t(ga) * d + k0 + kk] : 0.0;
-              Bt[kk * kEvTile + i] = gb < d ? A[size_t(gb) * d + k0 + kk] : 0.0;
+              Bt[kk * 2 * kEvTile + i] = in ? A[size_t(gb) * d + k0 + kk] : 0.0;
             }
           }
           __syncthreads();
@@ -170,8 +192,8 @@ __global__ void __launch_bounds__(kEvThreads) calib_evidence_kernel(CalibState s
           for (int k = 0; k < kEvNb; ++k) {
             const double2 a01 = *reinterpret_cast<const double2*>(At + k * kEvTile + ty * 4);
             const double2 a23 = *reinterpret_cast<const double2*>(At + k * kEvTile + ty * 4 + 2);
-            const double2 b01 = *reinterpret_cast<const double2*>(Bt + k * kEvTile + tx * 4);
-            const double2 b23 = *reinterpret_cast<const double2*>(Bt + k * kEvTile + tx * 4 + 2);
+            const double2 b01 = *reinterpret_cast<const double2*>(Bt + k * 2 * kEvTile + tx * 2);
+            const double2 b23 = *reinterpret_cast<const double2*>(Bt + k * 2 * kEvTile + kEvTile + tx * 2);
             const double a[4] = {a01.x, a01.y, a23.x, a23.y}, b[4] = {b01.x, b01.y, b23.x, b23.y};
 #pragma unroll
             for (int i = 0; i < 4; ++i)
@@ -184,8 +206,8 @@ __global__ void __launch_bounds__(kEvThreads) calib_evidence_kernel(CalibState s
             if (gi >= d) continue;
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-              const int gj = r0 + bj * kEvTile + tx * 4 + j;
-              if (gj <= gi) A[size_t(gi) * d + gj] -= acc[i][j];
+              const int gj = c0 + (j >> 1) * kEvTile + tx * 2 + (j & 1);
+              if (gj <= gi) A[size_t(gi) * d + gj] = cval[i][j] - acc[i][j];
             }
           }
           __syncthreads();
@@ -226,7 +248,7 @@ cudaError_t launch_calib_evidence(const base_layer_shape& s, const CalibState& s
   g.n = n_lambda;
   g.default_index = default_index;
   for (int i = 0; i < n_lambda; ++i) g.v[i] = lambdas[i];
-  const size_t smem = (size_t(3) * s.d + 2 * kEvNb * kEvTile) * sizeof(double);
+  const size_t smem = (size_t(3) * s.d + 3 * kEvNb * kEvTile) * sizeof(double);
   static size_t set_for = 0;
   if (smem > set_for) {
     cudaError_t a = cudaFuncSetAttribute(calib_evidence_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
