@@ -15,7 +15,7 @@ constexpr int kMaxVals = kMaxE / kWarp;
 constexpr int kMaxK = 16;
 constexpr int kMaxT = 1024;
 constexpr int kMaxSlots = 8192;     // T*K routed pairs held in shared memory by the routing kernel
-constexpr int kMaxSplit = 2;        // the down pass may split a tile's K range over up to this many work units
+constexpr int kMaxSplit = 4;        // the down pass may split a tile's K range over up to this many work units
 constexpr int kSegTokens = 128;     // tokens of one expert handled by one FFN work unit
 
 __device__ __forceinline__ float warp_sum(float v) {

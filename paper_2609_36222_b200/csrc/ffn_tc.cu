@@ -843,7 +843,9 @@ int choose_split(const base_layer_shape& s, int T, int budget, int ypair_copies)
   const int kb_all = s.I / kBlockK;
   const int expect_experts = std::min(std::min(budget, s.E), T * s.K);
   const int down_units = (s.d / 128) * expect_experts;
-  int want = down_units >= 2 * sm_count() ? 1 : kMaxSplit;
+  // two chunks when the down tiles alone cannot keep every SM busy twice over, four when even two chunks
+  // leave SMs without a unit (each further copy costs the combine about 1.5 us per 4 MB)
+  int want = down_units >= 2 * sm_count() ? 1 : (2 * down_units < sm_count() ? 4 : 2);
   while (want > 1 && (kb_all < 8 * want || want > ypair_copies)) want >>= 1;
   return want;
 }
@@ -918,8 +920,7 @@ cudaError_t launch_ffn_tc(const base_layer_shape& s, const base_layer_weights& w
   p.steps1 = (s.d / kBlockK + int(kKbPerStage) - 1) / int(kKbPerStage);
   // Few experts with long down rows (d/128 tiles each) leave SMs without a down unit and make every
   // down unit wait for the whole gate/up pass of its segment; the K range (I) is then cut into chunks
-  // of at least 8 k-blocks, as many as the workspace holds partial-sum copies for. (On Mixtral-sized
-  // experts two chunks and four measured within 2% of each other; more copies cost the combine more.)
+  // of at least 8 k-blocks, as many as the workspace holds partial-sum copies for (see choose_split).
   const int kb_all = s.I / kBlockK;
   p.ksplit = choose_split(s, T, budget, ws.ypair_copies);
   p.ypair_stride = ws.ypair_stride;
