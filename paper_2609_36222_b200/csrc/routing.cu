@@ -308,12 +308,21 @@ __device__ __forceinline__ void take_best(const uint32_t (&key)[NV], uint32_t& a
   if (gi != kNone && (gi & 31) == lane) avail &= ~(1u << (gi >> 5));
 }
 
+// A batch of at most kRoutingWarps tokens runs on ONE CTA (a warp per token): its "cluster" barrier is a
+// block barrier and nothing has to become visible to another SM between the stages.
+template <int kCtas>
 __device__ __forceinline__ void cluster_barrier() {
+  if (kCtas == 1) {
+    __syncthreads();
+    return;
+  }
   __threadfence();
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
+template <int kCtas>
 __device__ __forceinline__ uint32_t cluster_cta_rank() {
+  if (kCtas == 1) return 0;
   uint32_t r;
   asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
   return r;
@@ -332,7 +341,7 @@ __device__ __forceinline__ uint32_t cluster_cta_rank() {
 #define RT_STAMP(i)
 #endif
 
-template <int NV>
+template <int NV, int kCtas>
 __global__ void __launch_bounds__(kRoutingThreads) routing_kernel(RoutingArgs a) {
   const int T = a.T, E = a.E, K = a.K, S = T * K;
   extern __shared__ int32_t s_dyn[];   // [S] executed routes, then [chunks][E] per-expert token ballots
@@ -348,11 +357,11 @@ __global__ void __launch_bounds__(kRoutingThreads) routing_kernel(RoutingArgs a)
   __shared__ int16_t s_rank[kMaxE];
 
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int cta = int(cluster_cta_rank());
+  const int cta = int(cluster_cta_rank<kCtas>());
   const int gwarp = cta * kRoutingWarps + warp;
-  constexpr int kWarps = kClusterCtas * kRoutingWarps;
+  constexpr int kWarps = kCtas * kRoutingWarps;
   const int gthread = cta * kRoutingThreads + threadIdx.x;
-  constexpr int kAllThreads = kClusterCtas * kRoutingThreads;
+  constexpr int kAllThreads = kCtas * kRoutingThreads;
   if (threadIdx.x == 0) s_status = 0;
   pdl_wait();
   // The FFN kernel that follows starts on the early expert list below while this kernel is still
@@ -361,7 +370,7 @@ __global__ void __launch_bounds__(kRoutingThreads) routing_kernel(RoutingArgs a)
   // cannot start before every CTA of this kernel has passed launch_dependents.
   // (Done by the last CTA of the cluster, which has the fewest tokens to route, so that the device
   // fence below stays off the path to the selection.)
-  if (cta == kClusterCtas - 1) {
+  if (cta == kCtas - 1) {
     for (int i = threadIdx.x; i < a.max_segs * kMaxSplit; i += kRoutingThreads) a.ws.counters[kCtrReady + i] = 0;
     for (int e = threadIdx.x; e < E; e += kRoutingThreads) a.ws.gu_expert[e] = -1;   // "not yet known"
     if (threadIdx.x == 0) {
@@ -463,7 +472,7 @@ __global__ void __launch_bounds__(kRoutingThreads) routing_kernel(RoutingArgs a)
     }
   }
   RT_STAMP(1)
-  cluster_barrier();
+  cluster_barrier<kCtas>();
   RT_STAMP(2)
 
   // ---- 2: batch aggregation in the fixed order of aggregate_columns(). Every CTA sums all experts
@@ -617,7 +626,7 @@ __global__ void __launch_bounds__(kRoutingThreads) routing_kernel(RoutingArgs a)
     }
   }
   RT_STAMP(5)
-  cluster_barrier();
+  cluster_barrier<kCtas>();
   RT_STAMP(6)
 
   // ---- 4: dispatch lists, computed by every CTA from a shared-memory copy of the executed routes.
@@ -720,33 +729,33 @@ __global__ void __launch_bounds__(kRoutingThreads) routing_kernel(RoutingArgs a)
 
 constexpr size_t kRoutingMaxSmem = size_t(kMaxSlots) * 4 + size_t(kMaxT / 32) * kMaxE * 4;
 
-template <int NV>
+template <int NV, int kCtas>
 cudaError_t launch_routing_nv(const RoutingArgs& a, cudaLaunchConfig_t* cfg) {
-  static cudaError_t attr = cudaFuncSetAttribute(routing_kernel<NV>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  static cudaError_t attr = cudaFuncSetAttribute(routing_kernel<NV, kCtas>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                  int(kRoutingMaxSmem));
   if (attr != cudaSuccess) return attr;
-  return launch_pdl(routing_kernel<NV>, cfg->gridDim, cfg->blockDim, cfg->dynamicSmemBytes, cfg->stream, kClusterCtas, a);
+  return launch_pdl(routing_kernel<NV, kCtas>, cfg->gridDim, cfg->blockDim, cfg->dynamicSmemBytes, cfg->stream, kCtas, a);
 }
 
-cudaError_t launch_routing(const RoutingArgs& a, cudaStream_t st) {
+template <int kCtas>
+cudaError_t launch_routing_ctas(const RoutingArgs& a, cudaStream_t st) {
   cudaLaunchConfig_t cfg{};
-  cfg.gridDim = dim3(kClusterCtas);
+  cfg.gridDim = dim3(kCtas);
   cfg.blockDim = dim3(kRoutingThreads);
   cfg.dynamicSmemBytes = size_t(a.T) * a.K * 4 + size_t((a.T + 31) / 32) * a.E * 4;
   cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = kClusterCtas;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
   const int nv = (a.E + 31) / 32;
-  if (nv <= 1) return launch_routing_nv<1>(a, &cfg);
-  if (nv <= 2) return launch_routing_nv<2>(a, &cfg);
-  if (nv <= 4) return launch_routing_nv<4>(a, &cfg);
-  if (nv <= 8) return launch_routing_nv<8>(a, &cfg);
-  return launch_routing_nv<16>(a, &cfg);
+  if (nv <= 1) return launch_routing_nv<1, kCtas>(a, &cfg);
+  if (nv <= 2) return launch_routing_nv<2, kCtas>(a, &cfg);
+  if (nv <= 4) return launch_routing_nv<4, kCtas>(a, &cfg);
+  if (nv <= 8) return launch_routing_nv<8, kCtas>(a, &cfg);
+  return launch_routing_nv<16, kCtas>(a, &cfg);
+}
+
+cudaError_t launch_routing(const RoutingArgs& a, cudaStream_t st) {
+  // small batches: one warp per token fits one CTA, and block barriers replace the cluster's
+  if (a.T <= kRoutingWarps) return launch_routing_ctas<1>(a, st);
+  return launch_routing_ctas<kClusterCtas>(a, st);
 }
 
 // ------------------------------------------------------------------------------------------------
