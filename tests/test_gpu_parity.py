@@ -182,7 +182,9 @@ def test_shared_experts_added_by_a_second_call(out_dtype):
 
 # ------------------------------------------------------------------------------- edge cases
 
-@pytest.mark.parametrize("T", [1, 5, 33, 130, 256])
+# 16 / 17: last batch on the single-CTA routing kernel and first one on the cluster; 64 / 65 and 128 / 129: the
+# token-tile sizes of the FFN kernel and its dense / gathered gate-up pass
+@pytest.mark.parametrize("T", [1, 5, 16, 17, 33, 64, 65, 128, 129, 130, 256])
 def test_ragged_batch_sizes(T):
     cfg = wl.CONFIGS["qwen3"]
     small = wl.LayerConfig("qwen3_small", d=512, E=128, K=8, I=192, T=T, budgets=(16,))
