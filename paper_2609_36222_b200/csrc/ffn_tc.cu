@@ -33,8 +33,9 @@
 // programmatic-launch dependency. Larger batches gather the token rows into expert-sorted order
 // (epilogue warps, while the first weight boxes are already in flight) and use per-expert token tiles.
 //
-// Every wait is bounded: on expiry the CTA raises an abort flag, all roles leave their loops, TMEM
-// is freed and BASE_DEV_WAIT_EXPIRED is OR-ed into the status word.
+// Every wait is bounded: on expiry the CTA raises an abort flag, all roles leave their loops, the
+// producer lets its copies in flight land, TMEM is freed and BASE_DEV_WAIT_EXPIRED is OR-ed into the
+// status word.
 #include <cuda.h>
 
 #include <algorithm>
@@ -440,6 +441,14 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
       if (ok && mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1u, abort_flag)) {
         bars->stage_unit[stage].phase = 0;
         mbar_arrive(smem_u32(&bars->full[stage]));
+      }
+      if (!ok || *abort_flag) {
+        // A wait has expired somewhere in this CTA. Weight boxes of the last stages may still be on their
+        // way into shared memory, and a stage whose token box was never issued will not complete its
+        // barrier: give the copies in flight a fixed time to land (far above any load latency) before the
+        // CTA is allowed to give its shared memory back.
+        const long long t0 = clock64();
+        while (clock64() - t0 < 200000ll) __nanosleep(1000);   // about 100 us
       }
     }
     __syncwarp();
