@@ -128,6 +128,9 @@ __global__ void __launch_bounds__(kEvThreads) calib_evidence_kernel(CalibState s
       const int mrows = d - r0;
       if (mrows <= 0) break;
       // ---- panel: X = A21 L11^-T, row by row (one thread per row), and w_rest -= X w_k
+      // (the block is read through a volatile pointer: hoisting its 528 loads ahead of the substitution
+      // would spill the row)
+      const volatile double (*Dv)[kEvNb + 1] = D;
       for (int i = r0 + tid; i < d; i += kEvThreads) {
         double x[kEvNb];
         double* row = A + size_t(i) * d + k0;
@@ -138,8 +141,8 @@ __global__ void __launch_bounds__(kEvThreads) calib_evidence_kernel(CalibState s
         for (int j = 0; j < kEvNb; ++j) {
           double v = x[j];
 #pragma unroll
-          for (int c = 0; c < j; ++c) v -= x[c] * D[j][c];
-          v /= D[j][j];
+          for (int c = 0; c < j; ++c) v -= x[c] * Dv[j][c];
+          v /= Dv[j][j];
           x[j] = v;
           dot += v * w[k0 + j];
         }
