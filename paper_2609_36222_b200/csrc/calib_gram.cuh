@@ -150,19 +150,19 @@ gram_tc_kernel(const __grid_constant__ CUtensorMap map_hi, const __grid_constant
       if (!mbar_wait(smem_u32(&bars->acc_full[acc]), acc_phase, abort_flag, 64)) break;
       tcgen05_fence_after();
       const uint32_t taddr = tmem_base + (uint32_t(q4 * 32) << 16) + uint32_t(acc * 128);
-      float* g = p.gram + (size_t(u) * p.d + size_t(i) * 128 + q4 * 32 + lane) * p.d + size_t(j) * 128;
+      // A thread holds row r = q4*32 + lane of the tile, i.e. the sums over the tokens of z_r z_c for the tile's
+      // columns c. The Gram matrix is symmetric, so the value also belongs at [column][row]: written there, the
+      // 32 lanes of a warp touch 32 consecutive floats (one 128-byte line per instruction) instead of 32
+      // different rows. The mirror tile (j, i) is filled the same way by the unit that computes (i, j)^T.
+      // One element, one addition per launch, so the result does not depend on any order; the addition is
+      // done at the L2 and no load has to come back first.
+      float* g = p.gram + (size_t(u) * p.d + size_t(j) * 128) * p.d + size_t(i) * 128 + q4 * 32 + lane;
       for (int c0 = 0; c0 < 128; c0 += 16) {
         float v[16];
         tmem_ld16(taddr + c0, v);
 #pragma unroll
-        for (int c = 0; c < 16; c += 4) {
-          float4 o = *reinterpret_cast<const float4*>(g + c0 + c);
-          o.x += v[c];
-          o.y += v[c + 1];
-          o.z += v[c + 2];
-          o.w += v[c + 3];
-          *reinterpret_cast<float4*>(g + c0 + c) = o;
-        }
+        for (int c = 0; c < 16; ++c)
+          asm volatile("red.relaxed.gpu.global.add.f32 [%0], %1;" ::"l"(g + size_t(c0 + c) * p.d), "f"(v[c]) : "memory");
       }
       tcgen05_fence_before();
       mbar_arrive(smem_u32(&bars->acc_empty[acc]));
