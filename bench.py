@@ -466,8 +466,8 @@ def run_calibration(args, cfg, T):
         cal.reset()
         ms_acc = timed(lambda i: cal.accumulate(dl.weights, hids[i % n_b]), n_b * 4)
         ms_solve = timed(lambda i: cal.solve(1e-2), 1)
-        ms_select = timed(lambda i: cal.select_lambda(), 1)        # 25 candidates per expert, one Cholesky each
-        ms_solve_sel = timed(lambda i: cal.solve_selected(), 1)
+        ms_select = timed(lambda i: cal.select_lambda(), 1)        # 25 candidates per expert, one Cholesky each, + solution
+        ms_solve_sel = timed(lambda i: cal.solve_selected(), 1)    # the same solution by conjugate gradients
         ms_corr = timed(lambda i: cal.accumulate_correction(dl.weights, hids[i % n_b]), n_b * 4)
     A, b = cal.finalize()
     st = cal.statistics()
@@ -486,10 +486,10 @@ def run_calibration(args, cfg, T):
         "config": {"workload": f"{cfg.name} layer d={cfg.d} E={cfg.E} K={cfg.K} I={cfg.I}, calibration batches of {T} tokens",
                    "experts_with_pairs": active, "pairs_per_expert_max": float(n.max())},
         "parts_ms": {"layer_all_routes_plus_energy": ms_layer, "statistics": stat_ms, "ridge_solve_once": ms_solve,
-                     "lambda_by_evidence_25_candidates": ms_select, "ridge_solve_selected": ms_solve_sel,
+                     "lambda_by_evidence_25_candidates_and_solution": ms_select, "ridge_solve_selected_by_cg": ms_solve_sel,
                      "correction_batch": ms_corr},
-        "lambda_selection": {"fp64_flops": 25.0 * int((n > 1).sum()) * cfg.d ** 3 / 3.0,
-                             "tflops_fp64": 25.0 * int((n > 1).sum()) * cfg.d ** 3 / 3.0 / (ms_select * 1e-3) / 1e12,
+        "lambda_selection": {"fp64_flops": 26.0 * int((n > 1).sum()) * cfg.d ** 3 / 3.0,
+                             "tflops_fp64": 26.0 * int((n > 1).sum()) * cfg.d ** 3 / 3.0 / (ms_select * 1e-3) / 1e12,
                              "index_histogram": np.bincount(st["lambda_index"].cpu().numpy()[n > 1], minlength=25).tolist()},
         "cg_iterations": {"mean": float(iters[n > 0].mean()), "max": int(iters.max())},
         "roofline": {"bound": "hbm", "kernel": "gram_tc_kernel (with the transposes and vector statistics of the batch)",

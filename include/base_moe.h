@@ -277,8 +277,8 @@ int base_exact_removal_error(const base_layer_shape* shape, const base_layer_wei
  *   base_calib_reset(state)
  *   for every batch:  base_calib_accumulate(batch, state)             -- pass 1: statistics
  *   base_calib_solve(state, lambda)                                   -- a_u = (G_c + lambda I)^-1 q_c, b_u
- *     or: base_calib_select_lambda(state, grid) then base_calib_solve_selected(state)
- *                                                                     -- lambda per expert by marginal likelihood
+ *     or: base_calib_select_lambda(state, grid)                       -- lambda per expert by marginal likelihood,
+ *                                                                        and a_u, b_u for that lambda
  *   for every batch:  base_calib_accumulate_correction(batch, state)  -- pass 2: sum of exp(s-hat)
  *   base_calib_finalize(state, pred_A, pred_b)                        -- b_u += log(mean energy / mean exp(s-hat))
  *
@@ -305,9 +305,12 @@ int base_exact_removal_error(const base_layer_shape* shape, const base_layer_wei
  * eigendecomposition per expert, here each penalty takes one fp64 Cholesky factorisation, which yields
  * the same two quantities). The candidate of largest L (the first on a tie) becomes the expert's lambda;
  * a candidate for which the stored (fp32) Gram matrix makes G_c + lambda I indefinite gets L = -inf; an
- * expert with fewer than two pairs takes candidate n_lambda/2. solve_selected then solves every expert
- * with its own lambda. Its `workspace`: base_calib_select_workspace_bytes(shape) = E*d*d*8 bytes,
- * 256-byte aligned.
+ * expert with fewer than two pairs takes candidate n_lambda/2. The call also leaves the ridge solution for
+ * the chosen lambda in the state (a = L^-T L^-1 q_c from the factor of one more factorisation, b as above; cg_iters
+ * = 0), so the correction pass can follow directly. base_calib_solve_selected recomputes the same solution by
+ * conjugate gradients with every expert's own lambda (an independent route to the same numbers; slow when a small
+ * lambda leaves the system ill-conditioned). `workspace` of select_lambda: base_calib_select_workspace_bytes(shape)
+ * = E*d*d*8 bytes, 256-byte aligned.
  *
  * `state` is a caller-owned device buffer of base_calib_state_bytes(shape) bytes, 256-byte aligned,
  * holding in this order (each array 256-byte aligned): n, sum_y, sum_yy, sum_e, sum_p, coef_b

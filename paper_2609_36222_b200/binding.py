@@ -361,7 +361,8 @@ class Calibrator:
 
     def select_lambda(self, lambdas=None, stream=None):
         """Ridge penalty per expert by marginal likelihood over `lambdas` (default: the paper's grid, 25 values
-        logarithmically spaced from 1e-4 to 1e2); returns the grid. Follow with solve_selected()."""
+        logarithmically spaced from 1e-4 to 1e2) and the ridge solution for it; returns the grid.
+        (solve_selected() recomputes that solution by conjugate gradients.)"""
         if lambdas is None:
             lambdas = [1e-4 * (1e6 ** (i / 24.0)) for i in range(25)]
         lambdas = [float(v) for v in lambdas]

@@ -59,16 +59,20 @@ __global__ void __launch_bounds__(kEvThreads) calib_evidence_kernel(CalibState s
   double* Bt = At + kEvNb * kEvTile;   // [kEvNb][2 * kEvTile] ... of its column block (128 columns)
   __shared__ double D[kEvNb][kEvNb + 1];
   __shared__ double s_logsum;
-  __shared__ int s_pd;
+  __shared__ int s_pd, s_best;
   const int u = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const double n = st.n[u];
   double* ev_out = st.evidence + size_t(u) * kCalibMaxLambdas;
   if (n < 2.0) {
+    // nothing to judge by, and nothing to fit: a = 0, b = the one target (0 without a pair)
     if (tid == 0) {
       st.lambda_index[u] = grid.default_index;
       st.lambda[u] = grid.v[grid.default_index];
+      st.coef_b[u] = n >= 1.0 ? st.sum_y[u] / n : 0.0;
+      st.iters[u] = 0;
     }
     for (int i = tid; i < kCalibMaxLambdas; i += kEvThreads) ev_out[i] = 0.0;
+    for (int j = tid; j < d; j += kEvThreads) st.coef_a[size_t(u) * d + j] = 0.0;
     return;
   }
   const double sy = st.sum_y[u];
@@ -85,7 +89,11 @@ __global__ void __launch_bounds__(kEvThreads) calib_evidence_kernel(CalibState s
   double best = 0.0;
   int best_i = -1;
 
-  for (int li = 0; li < grid.n; ++li) {
+  // passes 0 .. n-1: the evidence of every candidate; pass n: the chosen candidate once more, this time
+  // keeping the factor, for the ridge solution a = L^-T (L^-1 q_c)
+  for (int pass = 0; pass <= grid.n; ++pass) {
+    const bool last = pass == grid.n;
+    const int li = last ? s_best : pass;
     const double lam = grid.v[li];
     // ---- A (lower triangle) = G - n m m^T + lambda I
     for (int i = warp; i < d; i += kEvThreads / 32) {
@@ -124,6 +132,12 @@ __global__ void __launch_bounds__(kEvThreads) calib_evidence_kernel(CalibState s
         wnorm2 += s2;
       }
       __syncthreads();
+      if (last) {   // the back substitution reads the factor from the scratch matrix
+        for (int idx = tid; idx < kEvNb * kEvNb; idx += kEvThreads) {
+          const int i = idx >> 5, j = idx & 31;
+          if (j <= i) A[size_t(k0 + i) * d + k0 + j] = D[i][j];
+        }
+      }
       const int r0 = k0 + kEvNb;
       const int mrows = d - r0;
       if (mrows <= 0) break;
@@ -217,6 +231,7 @@ __global__ void __launch_bounds__(kEvThreads) calib_evidence_kernel(CalibState s
         }
       }
     }
+    if (last) break;
     // ---- evidence of this penalty
     if (tid == 0) {
       double ev;
@@ -231,6 +246,7 @@ __global__ void __launch_bounds__(kEvThreads) calib_evidence_kernel(CalibState s
         best = ev;
         best_i = li;
       }
+      s_best = best_i;
     }
     __syncthreads();
   }
@@ -238,6 +254,63 @@ __global__ void __launch_bounds__(kEvThreads) calib_evidence_kernel(CalibState s
     for (int i = grid.n; i < kCalibMaxLambdas; ++i) ev_out[i] = 0.0;
     st.lambda_index[u] = best_i;
     st.lambda[u] = grid.v[best_i];
+    st.iters[u] = 0;
+  }
+  // ---- back substitution L^T a = w, block rows from the bottom up; a overwrites w in place
+  __syncthreads();
+  double* colsum = At;   // [warps][32] partial column sums
+  for (int k0 = d - kEvNb; k0 >= 0; k0 -= kEvNb) {
+    const int r0 = k0 + kEvNb;
+    // s_j = sum over the rows below of L[i][k0 + j] a[i]
+    double part[kEvNb];
+#pragma unroll
+    for (int j = 0; j < kEvNb; ++j) part[j] = 0.0;
+    for (int i = r0 + tid; i < d; i += kEvThreads) {
+      const double ai = w[i];
+      const double* row = A + size_t(i) * d + k0;
+#pragma unroll
+      for (int j = 0; j < kEvNb; ++j) part[j] = fma(row[j], ai, part[j]);
+    }
+#pragma unroll
+    for (int j = 0; j < kEvNb; ++j) {
+      double v = part[j];
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) v += __shfl_down_sync(0xffffffffu, v, o);
+      if (lane == 0) colsum[warp * kEvNb + j] = v;
+    }
+    for (int idx = tid; idx < kEvNb * kEvNb; idx += kEvThreads) {
+      const int i = idx >> 5, j = idx & 31;
+      D[i][j] = j <= i ? A[size_t(k0 + i) * d + k0 + j] : 0.0;
+    }
+    __syncthreads();
+    if (warp == 0) {
+      double sj = 0.0;
+      for (int wp = 0; wp < kEvThreads / 32; ++wp) sj += colsum[wp * kEvNb + lane];   // fixed order
+      double rhs = w[k0 + lane] - sj;
+      // upper-triangular solve with L11^T: lane = unknown, from the last one up
+      for (int j = kEvNb - 1; j >= 0; --j) {
+        const double aj = __shfl_sync(0xffffffffu, rhs, j) / D[j][j];
+        if (lane == j) w[k0 + j] = aj;
+        if (lane < j) rhs -= D[j][lane] * aj;
+      }
+    }
+    __syncthreads();
+  }
+  double dot = 0.0;
+  for (int j = tid; j < d; j += kEvThreads) {
+    const double aj = w[j];
+    st.coef_a[size_t(u) * d + j] = aj;
+    dot += aj * m[j];
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) dot += __shfl_down_sync(0xffffffffu, dot, o);
+  __syncthreads();
+  if (lane == 0) colsum[warp] = dot;
+  __syncthreads();
+  if (tid == 0) {
+    double t = 0.0;
+    for (int wp = 0; wp < kEvThreads / 32; ++wp) t += colsum[wp];
+    st.coef_b[u] = sy / n - t;
   }
 }
 

@@ -193,7 +193,10 @@ def test_lambda_by_evidence_matches_numpy_on_the_device_statistics(name, sizes, 
         else:
             assert st["lambda_index"][u] == int(np.argmax(ev))            # first maximum
         assert st["lambda"][u] == grid[st["lambda_index"][u]]
-    # the solve with the selected penalties: predictions on the expert's statistics against NumPy
+    # the ridge solution for the selected penalties, twice: left behind by the selection itself (from the Cholesky
+    # factor) and recomputed by conjugate gradients; both against NumPy on the expert's statistics
+    direct = {k: st[k].copy() for k in ("coef_a", "coef_b")}
+    assert not st["cg_iters"].any()
     cal.solve_selected()
     torch.cuda.synchronize()
     st2 = {k: v.cpu().numpy() for k, v in cal.statistics().items() if k != "gram"}
@@ -201,12 +204,21 @@ def test_lambda_by_evidence_matches_numpy_on_the_device_statistics(name, sizes, 
         n = float(st["n"][u])
         m = st["sum_z"][u] / n
         G = st["gram"][u].astype(np.float64)
-        Gc = 0.5 * (G + G.T) - n * np.outer(m, m)
+        Gl = np.tril(G) + np.tril(G, -1).T                                # what the factorisation reads
         qc = st["sum_yz"][u] - st["sum_y"][u] * m
-        a_ref = np.linalg.solve(Gc + st["lambda"][u] * np.eye(d), qc)
-        # compare through the quantity the fit minimises: a difference in a weighs by the Gram matrix
-        da = st2["coef_a"][u] - a_ref
-        assert da @ (Gc @ da) + st["lambda"][u] * (da @ da) <= 1e-10 * max(qc @ a_ref, 1e-30)
+        lam = st["lambda"][u]
+        for coef_a, coef_b, Gs in ((direct["coef_a"][u], direct["coef_b"][u], Gl),
+                                   (st2["coef_a"][u], st2["coef_b"][u], 0.5 * (G + G.T))):
+            Gc = Gs - n * np.outer(m, m)
+            a_ref = np.linalg.solve(Gc + lam * np.eye(d), qc)
+            # compare through the quantity the fit minimises: a difference in a weighs by the Gram matrix
+            da = coef_a - a_ref
+            assert da @ (Gc @ da) + lam * (da @ da) <= 1e-10 * max(qc @ a_ref, 1e-30)
+            assert abs(coef_b - (st["sum_y"][u] / n - a_ref @ m)) <= 1e-8 * (1 + abs(coef_b))
+    for u in range(E):                                                     # experts without a fit
+        if st["n"][u] < 2:
+            assert not direct["coef_a"][u].any()
+            assert direct["coef_b"][u] == (st["sum_y"][u] if st["n"][u] == 1 else 0.0)
 
 
 def test_lambda_by_evidence_end_to_end_against_the_oracle():
@@ -222,8 +234,7 @@ def test_lambda_by_evidence_end_to_end_against_the_oracle():
         lg = O.router_logits(h.z, base.router_w, base.router_bias)
         logits.append(lg)
         cal.accumulate(dl.weights, bits_to_device(h.hidden_bits, DEV), router_logits=torch.from_numpy(lg).to(DEV))
-    grid = np.array(cal.select_lambda())
-    cal.solve_selected()
+    grid = np.array(cal.select_lambda())                                   # leaves the solution for the chosen penalties
     for h, lg in zip(batches, logits):
         cal.accumulate_correction(dl.weights, bits_to_device(h.hidden_bits, DEV), router_logits=torch.from_numpy(lg).to(DEV))
     A_dev, b_dev = cal.finalize()
