@@ -7,6 +7,10 @@ input. Default workload: the Qwen3-30B-A3B-shaped layer, batch 64, expert budget
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
                     [--workload qwen3|mid|mixtral|tiny|qwen3_stack] [--budget M] [--batch T] [--sweep]
+                    [--bias-scale S] [--no-cpu] [--no-dense] [--profile] [--calib]
+
+--sweep prints one line per budget of the workload and a linear fit of step time against dispatched experts;
+--calib prints the line of the device calibration (statistics batches, ridge penalty selection, solves) instead.
 
 Prints ONE JSON line (rank 0). Timing: CUDA events on the launching stream around K graph
 replays; L2 is kept cold by rotating independently seeded weight replicas whose dispatched
