@@ -274,6 +274,38 @@ def base_moe_decode_layer_host(shape, weights, h_hidden, budget, h_out, workspac
     return h_out
 
 
+class HostLayerCall:
+    """base_moe_decode_layer_host with its arguments marshalled once, for a decode loop that reuses its buffers:
+    calling the object runs one step (blocks until h_out is written) and returns h_out. With joined=True (default)
+    the output and the n_dispatched word share one pinned host buffer, so they come back in a single copy."""
+
+    def __init__(self, shape, weights, h_hidden, budget, workspace, out_dtype=torch.bfloat16, gate_rule=GATE_PAPER,
+                 fill_rule=FILL_BACKFILL, ffn_impl=FFN_DEFAULT, stream=None, joined=True):
+        d, E, K, I = shape
+        T = h_hidden.shape[0]
+        assert not h_hidden.is_cuda and h_hidden.dtype == torch.bfloat16 and h_hidden.is_contiguous()
+        n_out = T * d * (4 if out_dtype == torch.float32 else 2)
+        if joined:
+            self._buf = torch.empty(n_out + 4, dtype=torch.uint8).pin_memory()
+            self.h_out = self._buf[:n_out].view(out_dtype).view(T, d)
+            self.h_n_dispatched = self._buf[n_out:].view(torch.int32)
+        else:
+            self.h_out = torch.empty(T, d, dtype=out_dtype).pin_memory()
+            self.h_n_dispatched = torch.zeros(1, dtype=torch.int32).pin_memory()
+        self._keep = (LayerShape(d, E, K, I), weights, h_hidden, workspace,
+                      LayerOptions(gate_rule, fill_rule, 1 if out_dtype == torch.float32 else 0, ffn_impl))
+        self._fn = lib().base_moe_decode_layer_host
+        self._args = (C.byref(self._keep[0]), C.byref(weights), h_hidden.data_ptr(), T, budget, self.h_out.data_ptr(),
+                      C.byref(self._keep[4]), self.h_n_dispatched.data_ptr(), workspace.data_ptr(), workspace.numel(),
+                      _stream(stream))
+
+    def __call__(self):
+        rc = self._fn(*self._args)
+        if rc != BASE_OK:
+            _check(rc)
+        return self.h_out
+
+
 def stack_workspace_bytes(d, E, K, I, T_max):
     n = lib().base_moe_decode_stack_workspace_bytes(C.byref(LayerShape(d, E, K, I)), T_max)
     if n == 0:

@@ -1,5 +1,6 @@
 // C-ABI entry points: argument checks, workspace carving, kernel sequencing. No device allocation,
 // no synchronisation (except the *_host entry point, which waits for its own copies).
+#include <cuda.h>
 #include <string.h>
 
 #include <mutex>
@@ -479,7 +480,30 @@ int base_moe_decode_layer_host(const base_layer_shape* shape, const base_layer_w
   char* io = static_cast<char*>(workspace) + ws.bytes;
   void* d_in = io;
   void* d_out = io + align_up(size_t(T) * shape->d * 2, 1024);
-  int32_t* d_nd = reinterpret_cast<int32_t*>(static_cast<char*>(d_out) + align_up(size_t(T) * shape->d * 4, 1024));
+  // When the caller's n_dispatched word sits right behind its output buffer, the device copies are laid out the
+  // same way and one copy brings both back.
+  const size_t out_bytes_h = size_t(T) * shape->d * ((opt && opt->out_is_fp32) ? 4 : 2);
+  bool joined = h_n_dispatched && reinterpret_cast<char*>(h_n_dispatched) == static_cast<char*>(h_out) + out_bytes_h;
+  if (joined) {
+    // adjacent addresses are not enough (two separate pinned allocations can touch): one copy may only span
+    // bytes of ONE allocation known to the driver
+    CUdeviceptr base = 0;
+    size_t size = 0;
+    const CUdeviceptr p = reinterpret_cast<CUdeviceptr>(h_out);
+    // (looked up through the runtime: the library must load on a machine without a driver)
+    typedef CUresult (*RangeFn)(CUdeviceptr*, size_t*, CUdeviceptr);
+    static RangeFn range_fn = [] {
+      void* f = nullptr;
+      cudaDriverEntryPointQueryResult q;
+      if (cudaGetDriverEntryPoint("cuMemGetAddressRange", &f, cudaEnableDefault, &q) != cudaSuccess ||
+          q != cudaDriverEntryPointSuccess)
+        f = nullptr;
+      return reinterpret_cast<RangeFn>(f);
+    }();
+    joined = range_fn && range_fn(&base, &size, p) == CUDA_SUCCESS && p + out_bytes_h + 4 <= base + size;
+  }
+  int32_t* d_nd = reinterpret_cast<int32_t*>(static_cast<char*>(d_out) +
+                                             (joined ? out_bytes_h : align_up(size_t(T) * shape->d * 4, 1024)));
   cudaError_t e = cudaMemcpyAsync(d_in, h_hidden_bf16, size_t(T) * shape->d * 2, cudaMemcpyHostToDevice, st);
   if (e != cudaSuccess) return cuda_fail(e);
   LayerCall c{};
@@ -495,9 +519,9 @@ int base_moe_decode_layer_host(const base_layer_shape* shape, const base_layer_w
   rc = enqueue_layer(c, ws, st, &launches);
   if (rc != BASE_OK) return rc;
   const size_t out_bytes = size_t(T) * shape->d * (c.opt.out_is_fp32 ? 4 : 2);
-  e = cudaMemcpyAsync(h_out, d_out, out_bytes, cudaMemcpyDeviceToHost, st);
+  e = cudaMemcpyAsync(h_out, d_out, out_bytes + (joined ? 4 : 0), cudaMemcpyDeviceToHost, st);
   if (e != cudaSuccess) return cuda_fail(e);
-  if (h_n_dispatched) {
+  if (h_n_dispatched && !joined) {
     e = cudaMemcpyAsync(h_n_dispatched, d_nd, 4, cudaMemcpyDeviceToHost, st);
     if (e != cudaSuccess) return cuda_fail(e);
   }

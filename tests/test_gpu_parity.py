@@ -317,6 +317,18 @@ def test_host_entry_point_matches_device_entry_point(layers):
     torch.cuda.synchronize()
     assert torch.equal(h_out, dev_out.cpu())
     assert 0 < nd.item() <= 32
+    # the prepared call (arguments marshalled once; result and count in one pinned buffer, one copy back)
+    for joined in (True, False):
+        call = B.HostLayerCall(dl.shape, dl.weights, h_in, 32, ws, joined=joined)
+        call.h_out.zero_()
+        call.h_n_dispatched.zero_()
+        assert torch.equal(call(), dev_out.cpu())
+        assert call.h_n_dispatched.item() == nd.item()
+    call = B.HostLayerCall(dl.shape, dl.weights, h_in, 32, ws, out_dtype=torch.float32)
+    out32 = torch.empty(cfg.T, cfg.d, dtype=torch.float32, device=DEV)
+    dl.run(bits_to_device(host.hidden_bits, DEV), 32, out=out32)
+    torch.cuda.synchronize()
+    assert torch.equal(call(), out32.cpu()) and call.h_n_dispatched.item() == nd.item()
 
 
 def test_stack_teacher_forced_and_chained():
