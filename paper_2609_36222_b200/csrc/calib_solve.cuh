@@ -64,16 +64,26 @@ __global__ void __launch_bounds__(kSolveThreads) calib_solve_kernel(CalibState s
     part = 0.0;
     for (int j = threadIdx.x; j < d; j += kSolveThreads) part += m[j] * pv[j];
     const double mp = block_sum(part, s_red);
-    for (int row = warp; row < d; row += kSolveThreads / 32) {
-      const float* g = G + size_t(row) * d;
-      double acc = 0.0;
+    // four rows per warp and step: the direction's four values are read from shared memory once for all of
+    // them (that read, not the matrix, limited the product), and four matrix loads are in flight per lane
+    for (int row0 = warp * 4; row0 < d; row0 += kSolveThreads / 32 * 4) {
+      const float* g = G + size_t(row0) * d;
+      double acc[4] = {0.0, 0.0, 0.0, 0.0};
       for (int c = lane * 4; c < d; c += 128) {
-        const float4 gv = *reinterpret_cast<const float4*>(g + c);
-        acc += double(gv.x) * pv[c] + double(gv.y) * pv[c + 1] + double(gv.z) * pv[c + 2] + double(gv.w) * pv[c + 3];
+        const double p0 = pv[c], p1 = pv[c + 1], p2 = pv[c + 2], p3 = pv[c + 3];
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+          const float4 gv = *reinterpret_cast<const float4*>(g + size_t(r) * d + c);
+          acc[r] += double(gv.x) * p0 + double(gv.y) * p1 + double(gv.z) * p2 + double(gv.w) * p3;
+        }
       }
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) acc += __shfl_down_sync(0xffffffffu, acc, o);
-      if (lane == 0) ap[row] = acc - n * m[row] * mp + lambda * pv[row];
+      for (int r = 0; r < 4; ++r) {
+        double a = acc[r];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) a += __shfl_down_sync(0xffffffffu, a, o);
+        if (lane == 0) ap[row0 + r] = a - n * m[row0 + r] * mp + lambda * pv[row0 + r];
+      }
     }
     __syncthreads();
     part = 0.0;
