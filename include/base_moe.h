@@ -220,6 +220,12 @@ int base_moe_decode_layer_host(const base_layer_shape* shape, const base_layer_w
                                const void* h_hidden_bf16, int T, int budget, void* h_out,
                                const base_layer_options* opt, int32_t* h_n_dispatched,
                                void* workspace, size_t workspace_bytes, void* stream);
+/* The same, enqueued only: nothing is waited for, h_out is valid once `stream` has passed the call. With pinned
+ * host buffers the whole step (copy in, four kernels, copy out) can be captured into a CUDA graph by the caller. */
+int base_moe_decode_layer_host_enqueue(const base_layer_shape* shape, const base_layer_weights* weights,
+                                       const void* h_hidden_bf16, int T, int budget, void* h_out,
+                                       const base_layer_options* opt, int32_t* h_n_dispatched,
+                                       void* workspace, size_t workspace_bytes, void* stream);
 
 /*
  * L layers back to back on one stream (the full-model decode-step workload). Layer l reads

@@ -27,6 +27,7 @@ DEV_NONFINITE_SCORE, DEV_WAIT_EXPIRED, DEV_BAD_INDEX = 1, 2, 4
 EXPORTS = (
     "base_predict_costs", "base_aggregate_select", "base_moe_decode_layer_workspace_bytes",
     "base_moe_decode_layer", "base_moe_decode_layer_noalloc", "base_moe_decode_layer_host_workspace_bytes", "base_moe_decode_layer_host",
+    "base_moe_decode_layer_host_enqueue",
     "base_moe_decode_stack_workspace_bytes", "base_moe_decode_stack", "base_profile_events",
     "base_last_launch_count", "base_true_removal_costs", "base_energy_retained", "base_exact_removal_error",
     "base_calib_state_bytes", "base_calib_workspace_bytes", "base_calib_reset", "base_calib_accumulate",
@@ -85,6 +86,7 @@ def lib():
     L.base_moe_decode_layer_host_workspace_bytes.restype = C.c_size_t
     L.base_moe_decode_layer_host.argtypes = [C.POINTER(LayerShape), C.POINTER(LayerWeights), vp, ip, ip, vp,
                                              C.POINTER(LayerOptions), vp, vp, C.c_size_t, vp]
+    L.base_moe_decode_layer_host_enqueue.argtypes = L.base_moe_decode_layer_host.argtypes
     L.base_moe_decode_stack_workspace_bytes.argtypes = [C.POINTER(LayerShape), ip]
     L.base_moe_decode_stack_workspace_bytes.restype = C.c_size_t
     L.base_moe_decode_stack.argtypes = [C.POINTER(LayerShape), C.POINTER(LayerWeights), ip, vp, ip, ip, vp,
@@ -277,10 +279,11 @@ def base_moe_decode_layer_host(shape, weights, h_hidden, budget, h_out, workspac
 class HostLayerCall:
     """base_moe_decode_layer_host with its arguments marshalled once, for a decode loop that reuses its buffers:
     calling the object runs one step (blocks until h_out is written) and returns h_out. With joined=True (default)
-    the output and the n_dispatched word share one pinned host buffer, so they come back in a single copy."""
+    the output and the n_dispatched word share one pinned host buffer, so they come back in a single copy; with
+    graph=True the step is one CUDA-graph launch."""
 
     def __init__(self, shape, weights, h_hidden, budget, workspace, out_dtype=torch.bfloat16, gate_rule=GATE_PAPER,
-                 fill_rule=FILL_BACKFILL, ffn_impl=FFN_DEFAULT, stream=None, joined=True):
+                 fill_rule=FILL_BACKFILL, ffn_impl=FFN_DEFAULT, stream=None, joined=True, graph=False):
         d, E, K, I = shape
         T = h_hidden.shape[0]
         assert not h_hidden.is_cuda and h_hidden.dtype == torch.bfloat16 and h_hidden.is_contiguous()
@@ -298,8 +301,28 @@ class HostLayerCall:
         self._args = (C.byref(self._keep[0]), C.byref(weights), h_hidden.data_ptr(), T, budget, self.h_out.data_ptr(),
                       C.byref(self._keep[4]), self.h_n_dispatched.data_ptr(), workspace.data_ptr(), workspace.numel(),
                       _stream(stream))
+        self._graph = None
+        if graph:
+            # graph=True: copy in, the four kernels and copy out are captured once (through the enqueue-only entry
+            # point, on a stream of their own) and a step is one graph launch plus the wait for it. h_hidden must
+            # be pinned. The first, ordinary call sets up what must not happen inside a capture.
+            assert h_hidden.is_pinned()
+            self()
+            self._gstream = torch.cuda.Stream(device=workspace.device)
+            args = self._args[:-1] + (self._gstream.cuda_stream,)
+            self._graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(self._graph, stream=self._gstream):
+                rc = lib().base_moe_decode_layer_host_enqueue(*args)
+            if rc != BASE_OK:
+                self._graph = None
+                _check(rc)
 
     def __call__(self):
+        if self._graph is not None:
+            with torch.cuda.stream(self._gstream):
+                self._graph.replay()
+            self._gstream.synchronize()
+            return self.h_out
         rc = self._fn(*self._args)
         if rc != BASE_OK:
             _check(rc)

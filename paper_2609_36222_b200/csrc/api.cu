@@ -467,10 +467,9 @@ size_t base_moe_decode_layer_host_workspace_bytes(const base_layer_shape* shape,
   return carve_workspace(nullptr, *shape, T_max).bytes + io;
 }
 
-int base_moe_decode_layer_host(const base_layer_shape* shape, const base_layer_weights* weights,
-                               const void* h_hidden_bf16, int T, int budget, void* h_out,
-                               const base_layer_options* opt, int32_t* h_n_dispatched, void* workspace,
-                               size_t workspace_bytes, void* stream) {
+static int layer_host(const base_layer_shape* shape, const base_layer_weights* weights, const void* h_hidden_bf16,
+                      int T, int budget, void* h_out, const base_layer_options* opt, int32_t* h_n_dispatched,
+                      void* workspace, size_t workspace_bytes, void* stream, bool wait) {
   int rc = check_layer_args(shape, weights, h_hidden_bf16, nullptr, T, budget, opt);
   if (rc != BASE_OK) return rc;
   if (!h_out || !workspace || (reinterpret_cast<uintptr_t>(workspace) & 1023u)) return BASE_ERR_INVALID_ARG;
@@ -525,10 +524,28 @@ int base_moe_decode_layer_host(const base_layer_shape* shape, const base_layer_w
     e = cudaMemcpyAsync(h_n_dispatched, d_nd, 4, cudaMemcpyDeviceToHost, st);
     if (e != cudaSuccess) return cuda_fail(e);
   }
-  e = cudaStreamSynchronize(st);
-  if (e != cudaSuccess) return cuda_fail(e);
+  if (wait) {
+    e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail(e);
+  }
   g_last_launches = launches;
   return BASE_OK;
+}
+
+int base_moe_decode_layer_host(const base_layer_shape* shape, const base_layer_weights* weights,
+                               const void* h_hidden_bf16, int T, int budget, void* h_out,
+                               const base_layer_options* opt, int32_t* h_n_dispatched, void* workspace,
+                               size_t workspace_bytes, void* stream) {
+  return layer_host(shape, weights, h_hidden_bf16, T, budget, h_out, opt, h_n_dispatched, workspace, workspace_bytes,
+                    stream, true);
+}
+
+int base_moe_decode_layer_host_enqueue(const base_layer_shape* shape, const base_layer_weights* weights,
+                                       const void* h_hidden_bf16, int T, int budget, void* h_out,
+                                       const base_layer_options* opt, int32_t* h_n_dispatched, void* workspace,
+                                       size_t workspace_bytes, void* stream) {
+  return layer_host(shape, weights, h_hidden_bf16, T, budget, h_out, opt, h_n_dispatched, workspace, workspace_bytes,
+                    stream, false);
 }
 
 size_t base_moe_decode_stack_workspace_bytes(const base_layer_shape* shape, int T_max) {

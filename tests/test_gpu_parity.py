@@ -324,6 +324,12 @@ def test_host_entry_point_matches_device_entry_point(layers):
         call.h_n_dispatched.zero_()
         assert torch.equal(call(), dev_out.cpu())
         assert call.h_n_dispatched.item() == nd.item()
+    call = B.HostLayerCall(dl.shape, dl.weights, h_in, 32, ws, graph=True)      # one graph launch per step
+    for _ in range(3):
+        call.h_out.zero_()
+        call.h_n_dispatched.zero_()
+        assert torch.equal(call(), dev_out.cpu())
+        assert call.h_n_dispatched.item() == nd.item()
     call = B.HostLayerCall(dl.shape, dl.weights, h_in, 32, ws, out_dtype=torch.float32)
     out32 = torch.empty(cfg.T, cfg.d, dtype=torch.float32, device=DEV)
     dl.run(bits_to_device(host.hidden_bits, DEV), 32, out=out32)
