@@ -7,10 +7,11 @@ input. Default workload: the Qwen3-30B-A3B-shaped layer, batch 64, expert budget
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
                     [--workload qwen3|mid|mixtral|tiny|qwen3_stack] [--budget M] [--batch T] [--sweep]
-                    [--bias-scale S] [--no-cpu] [--no-dense] [--profile] [--calib]
+                    [--bias-scale S] [--no-cpu] [--no-dense] [--profile] [--calib] [--ablation]
 
 --sweep prints one line per budget of the workload and a linear fit of step time against dispatched experts;
---calib prints the line of the device calibration (statistics batches, ridge penalty selection, solves) instead.
+--calib prints the line of the device calibration (statistics batches, ridge penalty selection, solves) instead;
+--ablation the retained energy of the selection-score variants on a planted workload.
 
 Prints ONE JSON line (rank 0). Timing: CUDA events on the launching stream around K graph
 replays; L2 is kept cold by rotating independently seeded weight replicas whose dispatched
@@ -503,6 +504,61 @@ def run_calibration(args, cfg, T):
     print(json.dumps(line))
 
 
+def run_ablation(args, cfg):
+    """Extra line (not the headline): retained energy ER(m) (Eq. energy_retained) of the selection scores of
+    App. Selection-Rule Ablation on a PLANTED synthetic workload -- the structure of the paper's table, not its
+    numbers: every expert's gate matrix gets a seeded rank-one term, so that its output energy depends on the
+    token's direction and a predictor has something to learn. The predictor is calibrated on the device
+    (statistics, ridge penalty by marginal likelihood, correction) on calibration batches and every rule is then
+    scored on held-out batches against the true removal costs of the same batches."""
+    import torch
+    from paper_2609_36222_b200 import binding as B, workloads as wl
+    from paper_2609_36222_b200.layer import DeviceLayer, bits_to_device
+    dev = torch.device("cuda:0")
+    torch.cuda.set_device(dev)
+    alpha, T_cal, n_cal, T_eval, n_eval = args.planted_alpha, 256, 16, cfg.T, 8
+    dl = DeviceLayer(cfg, dev, T_max=max(T_cal, T_eval))
+    v = wl.normal_f64(wl.stream_key(0, cfg.name, 0, "planted_v"), 0, cfg.E * cfg.d).reshape(cfg.E, cfg.d)
+    v /= np.linalg.norm(v, axis=1, keepdims=True)
+    wg = dl.tensors["w_gate"]
+    wg.copy_((wg.float() + alpha * torch.from_numpy(v).to(dev).float()[:, None, :]).to(torch.bfloat16))
+    cal = B.Calibrator(dl.shape, T_cal, dev)
+    cal_batches = [bits_to_device(wl.hidden_bits(cfg, T_cal, 0, 300 + i), dev) for i in range(n_cal)]
+    t0 = time.perf_counter()
+    for h in cal_batches:
+        cal.accumulate(dl.weights, h)
+    cal.select_lambda()
+    for h in cal_batches:
+        cal.accumulate_correction(dl.weights, h)
+    A, b = cal.finalize()
+    torch.cuda.synchronize()
+    t_cal = time.perf_counter() - t0
+    dl.tensors["pred_A"], dl.tensors["pred_b"] = A, b
+    dl.weights = B.make_weights(dl.tensors)
+    rules = {"predicted (BASE)": B.SCORE_PREDICTED, "sum w^2": B.SCORE_WEIGHT_SQ, "sum w": B.SCORE_WEIGHT,
+             "static energy": B.SCORE_STATIC, "top-1 union": B.SCORE_TOP1_UNION}
+    budgets = [m for m in cfg.budgets if m < cfg.E]
+    table = {name: {str(m): 0.0 for m in budgets} for name in rules}
+    out = torch.empty(T_eval, cfg.d, dtype=torch.float32, device=dev)
+    for i in range(n_eval):
+        hid = bits_to_device(wl.hidden_bits(cfg, T_eval, 0, 900 + i), dev)
+        true_costs, _, _, _ = B.base_true_removal_costs(dl.shape, dl.weights, hid, dl.workspace)
+        for m in budgets:
+            d_star, _, _ = B.base_aggregate_select(true_costs, m)
+            for name, rule in rules.items():
+                dbg, dt = B.alloc_debug(T_eval, cfg.E, cfg.K, m, dev)
+                B.base_moe_decode_layer(dl.shape, dl.weights, hid, m, out, dl.workspace, debug=dbg, score_rule=rule)
+                table[name][str(m)] += float(B.base_energy_retained(d_star, dt["active_mask"], m).cpu()[0]) / n_eval
+    idx = cal.statistics()["lambda_index"].cpu().numpy()
+    print(json.dumps({
+        "metric": "retained_energy_by_selection_rule", "unit": "ER(m), 1 = the oracle active set", "n_gpus": 1,
+        "data": "synthetic, planted energy direction (alpha = %g)" % alpha,
+        "config": {"workload": f"{cfg.name} layer d={cfg.d} E={cfg.E} K={cfg.K} I={cfg.I}, {n_eval} held-out batches of "
+                               f"{T_eval} tokens, predictor calibrated on {n_cal} x {T_cal} tokens on the device"},
+        "retained_energy": table, "calibration_s": t_cal,
+        "lambda_index_histogram": np.bincount(idx, minlength=25).tolist()}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -523,6 +579,10 @@ def main():
     ap.add_argument("--bias-scale", type=float, default=1.0,
                     help="scale of the Zipf router bias (1 = the workload as defined; 0 = flat routing, a sensitivity "
                          "row that is not one of the defined configurations)")
+    ap.add_argument("--planted-alpha", type=float, default=3.0,
+                    help="--ablation: weight of the rank-one term planted in every expert's gate matrix")
+    ap.add_argument("--ablation", action="store_true",
+                    help="retained energy of the selection-score variants on a planted workload (extra line)")
     ap.add_argument("--calib", action="store_true",
                     help="extra line: device calibration of the predictor on the workload's layer shape")
     args = ap.parse_args()
@@ -551,6 +611,8 @@ def main():
                               "expert_bytes": cfg.expert_bytes}))
     elif args.calib:
         run_calibration(args, cfg, args.batch or 1024)
+    elif args.ablation:
+        run_ablation(args, cfg)
     elif args.impl == "reference":
         run_reference(args, cfg, T, M)
     else:
