@@ -539,6 +539,7 @@ def run_ablation(args, cfg):
              "static energy": B.SCORE_STATIC, "top-1 union": B.SCORE_TOP1_UNION}
     budgets = [m for m in cfg.budgets if m < cfg.E]
     table = {name: {str(m): 0.0 for m in budgets} for name in rules}
+    cross = {str(m): [0.0, 0.0] for m in budgets}      # exact error of the BASE set and its individual (additive) part
     out = torch.empty(T_eval, cfg.d, dtype=torch.float32, device=dev)
     for i in range(n_eval):
         hid = bits_to_device(wl.hidden_bits(cfg, T_eval, 0, 900 + i), dev)
@@ -549,13 +550,19 @@ def run_ablation(args, cfg):
                 dbg, dt = B.alloc_debug(T_eval, cfg.E, cfg.K, m, dev)
                 B.base_moe_decode_layer(dl.shape, dl.weights, hid, m, out, dl.workspace, debug=dbg, score_rule=rule)
                 table[name][str(m)] += float(B.base_energy_retained(d_star, dt["active_mask"], m).cpu()[0]) / n_eval
+                if rule == B.SCORE_PREDICTED:   # Eq. error_decomposition: how much of the exact error the additive estimate misses
+                    ex = B.base_exact_removal_error(dl.shape, dl.weights, hid, dt["active_mask"], dl.workspace).cpu().numpy()
+                    cross[str(m)][0] += float(ex[0])
+                    cross[str(m)][1] += float(ex[1])
     idx = cal.statistics()["lambda_index"].cpu().numpy()
     print(json.dumps({
         "metric": "retained_energy_by_selection_rule", "unit": "ER(m), 1 = the oracle active set", "n_gpus": 1,
         "data": "synthetic, planted energy direction (alpha = %g)" % alpha,
         "config": {"workload": f"{cfg.name} layer d={cfg.d} E={cfg.E} K={cfg.K} I={cfg.I}, {n_eval} held-out batches of "
                                f"{T_eval} tokens, predictor calibrated on {n_cal} x {T_cal} tokens on the device"},
-        "retained_energy": table, "calibration_s": t_cal,
+        "retained_energy": table,
+        "exact_over_additive_error_of_the_base_set": {m: (v[0] / v[1] if v[1] > 0 else None) for m, v in cross.items()},
+        "calibration_s": t_cal,
         "lambda_index_histogram": np.bincount(idx, minlength=25).tolist()}))
 
 
