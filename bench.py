@@ -6,7 +6,7 @@ SwiGLU FFN over the dispatched experts, combine) over one decode batch of synthe
 input. Default workload: the Qwen3-30B-A3B-shaped layer, batch 64, expert budget 32.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                    [--workload qwen3|mid|mixtral|tiny|qwen3_stack] [--budget M] [--batch T] [--sweep]
+                    [--workload qwen3|mid|mixtral|tiny|qwen3_stack|dsv2lite|qwen15moe] [--budget M] [--batch T] [--sweep]
                     [--bias-scale S] [--no-cpu] [--no-dense] [--profile] [--calib] [--ablation]
 
 --sweep prints one line per budget of the workload and a linear fit of step time against dispatched experts;
@@ -146,12 +146,12 @@ def oracle_step_seconds(cfg, T, M, repeats, layer=0):
 
     # materialise the inputs (not timed: they are the workload, not the method)
     logits0 = O.router_logits(z, rw, rb)
-    res = O.moe_decode_layer(z, logits0, A, pb, ew, cfg.K, M)
+    res = O.moe_decode_layer(z, logits0, A, pb, ew, cfg.K, M, router_norm=cfg.router_norm)
     times = []
     for _ in range(repeats):
         t0 = time.perf_counter()
         logits = O.router_logits(z, rw, rb)
-        res = O.moe_decode_layer(z, logits, A, pb, ew, cfg.K, M)
+        res = O.moe_decode_layer(z, logits, A, pb, ew, cfg.K, M, router_norm=cfg.router_norm)
         times.append(time.perf_counter() - t0)
     try:
         from threadpoolctl import threadpool_info
@@ -241,7 +241,8 @@ def run_ours(args, cfg, T, M):
                                     n_dispatched=nd_buf, stream=stream)
         else:
             r = i % n_rep
-            B.base_moe_decode_layer(shape, layers[r].weights, hidden[r], budget, out, ws, debug=dbgs[r], stream=stream)
+            B.base_moe_decode_layer(shape, layers[r].weights, hidden[r], budget, out, ws, debug=dbgs[r], stream=stream,
+                                    router_norm=cfg.router_norm)
 
     # one eager pass (also fills n_dispatched per replica), then capture one graph per replica
     with torch.cuda.stream(stream):

@@ -49,6 +49,7 @@ class LayerConfig:
     budgets: tuple
     layers: int = 1
     batches: tuple = field(default_factory=tuple)  # stack sweep only
+    router_norm: int = 0   # 0: router weights renormalised over the top-K; 1: plain softmax over all experts
 
     @property
     def expert_bytes(self) -> int:
@@ -62,6 +63,11 @@ CONFIGS = {
     "qwen3_stack": LayerConfig("qwen3_stack", d=2048, E=128, K=8, I=768, T=64, budgets=(16, 32, 64),
                                layers=48, batches=(1, 8, 32, 64, 128, 256)),
     "mixtral": LayerConfig("mixtral", d=4096, E=8, K=2, I=14336, T=128, budgets=(2, 4, 6, 8)),
+    # The paper's two other models, routed experts only (their always-on shared experts are outside the selection,
+    # Sec. 3.1). The paper gives expert counts and top-K; widths are those of the public model configurations
+    # (hidden 2048, expert intermediate 1408 for both); neither renormalises the top-K router weights.
+    "dsv2lite": LayerConfig("dsv2lite", d=2048, E=64, K=6, I=1408, T=64, budgets=(8, 16, 24, 32, 64), router_norm=1),
+    "qwen15moe": LayerConfig("qwen15moe", d=2048, E=60, K=4, I=1408, T=64, budgets=(8, 16, 24, 32, 60), router_norm=1),
 }
 CONFIG_ORDER = ("tiny", "mid", "qwen3", "qwen3_stack", "mixtral")
 

@@ -105,6 +105,18 @@ def test_simple_and_tensor_core_ffn_agree(layers):
     assert d <= 2e-3 * np.abs(a["got"]["y"]).max()
 
 
+@pytest.mark.parametrize("name", ["dsv2lite", "qwen15moe"])
+def test_other_models_at_their_bench_shapes(name):
+    """The two other models of Sec. 4.1 at the widths bench.py times them with (hidden 2048, expert intermediate
+    1408, batch 64), router weights not renormalised over the top-K, at a tight and at the unlimited budget."""
+    cfg = wl.CONFIGS[name]
+    host = HostLayer(cfg)
+    dl = device_layer_from_host(host, DEV)
+    for M in (16, cfg.E):
+        rep = check_layer(host, dl, M, router_norm=cfg.router_norm)
+    assert (rep["ref"]["w"].sum(axis=1) < 1.0).all()
+
+
 @pytest.mark.parametrize("E,K,T", [(60, 4, 24), (64, 6, 48), (60, 4, 100)])
 def test_other_model_shapes(E, K, T):
     """Expert counts and top-K of the paper's other two models (Sec. 4.1: 60 experts with K = 4 -- not a
