@@ -125,8 +125,9 @@ def ffn_algorithmic_bytes(cfg, T, n_dispatched):
 
 # ------------------------------------------------------------------------------------------ oracle arm
 
-def oracle_step_seconds(cfg, T, M, repeats, layer=0):
-    """Time the CPU oracle, as it stands, on one full step of the workload. Returns (best seconds, cores)."""
+def oracle_step_seconds(cfg, T, M, repeats, layer=0, warmup=0, budget_s=None, mean=False):
+    """Time the CPU oracle, as it stands, on full steps of the workload: `warmup` untimed steps, then up to `repeats`
+    timed ones (fewer when budget_s seconds are used up). Returns (best or mean seconds, cores, n_dispatched, steps timed)."""
     from oracle import base_oracle as O
     from paper_2609_36222_b200 import workloads as wl
 
@@ -148,34 +149,40 @@ def oracle_step_seconds(cfg, T, M, repeats, layer=0):
     logits0 = O.router_logits(z, rw, rb)
     res = O.moe_decode_layer(z, logits0, A, pb, ew, cfg.K, M, router_norm=cfg.router_norm)
     times = []
-    for _ in range(repeats):
+    t_begin = time.perf_counter()
+    for i in range(warmup + repeats):
         t0 = time.perf_counter()
         logits = O.router_logits(z, rw, rb)
         res = O.moe_decode_layer(z, logits, A, pb, ew, cfg.K, M, router_norm=cfg.router_norm)
-        times.append(time.perf_counter() - t0)
+        if i >= warmup:
+            times.append(time.perf_counter() - t0)
+        if budget_s is not None and times and time.perf_counter() - t_begin > budget_s:
+            break
     try:
         from threadpoolctl import threadpool_info
         cores = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
     except Exception:
         cores = os.cpu_count() or 1
-    return min(times), cores, res["n_dispatched"]
+    return (sum(times) / len(times) if mean else min(times)), cores, res["n_dispatched"], len(times)
 
 
 def run_reference(args, cfg, T, M):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    reps = max(1, min(args.steps, 3))
-    best, cores, nd = oracle_step_seconds(cfg, T, M, reps)
-    us = best * 1e6
+    # W warm-up steps and K timed steps like the CUDA arm, each a full step of the workload on replica 0; the run is
+    # cut off after about a minute of oracle time, and the line says how many steps were timed
+    warm = max(0, min(args.warmup, 3))
+    sec, cores, nd, reps = oracle_step_seconds(cfg, T, M, max(1, args.steps), warmup=warm, budget_s=60.0, mean=True)
+    us = sec * 1e6
     line = {
         "impl": "reference", "metric": "moe_decode_layer_us_per_step", "value": us, "unit": "us/step",
-        "n_gpus": args.gpus, "steps": reps, "warmup": 1, "ms_per_step": us / 1e3, "higher_is_better": False,
+        "n_gpus": args.gpus, "steps": reps, "warmup": warm, "ms_per_step": us / 1e3, "higher_is_better": False,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": f"{cfg.name} layer d={cfg.d} E={cfg.E} K={cfg.K} I={cfg.I} batch={T} budget={M}",
                    "n_dispatched": nd},
         "cpu_baseline": {"value": us, "unit": "us/step", "cores": cores, "kind": "oracle",
-                         "sample": f"{reps} full step(s) of the workload (replica 0), best of {reps}"},
+                         "sample": f"mean of {reps} full step(s) of the workload (replica 0) after {warm} warm-up step(s)"},
         "e2e": {"value": us, "unit": "us/step", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -425,7 +432,7 @@ def run_ours(args, cfg, T, M):
     # CPU baseline: the oracle, as it stands, on this machine's host cores
     if not args.no_cpu and not args.profile:
         reps = 2 if cfg.expert_bytes < (64 << 20) else 1
-        best, cores, _ = oracle_step_seconds(cfg if not stack else wl.CONFIGS["qwen3"], T, M, reps)
+        best, cores, _, _ = oracle_step_seconds(cfg if not stack else wl.CONFIGS["qwen3"], T, M, reps)
         scale = cfg.layers if stack else 1
         line["cpu_baseline"] = {"value": best * 1e6 * scale, "unit": "us/step", "cores": cores, "kind": "oracle",
                                 "sample": f"{reps} full layer step(s), best of {reps}" +
