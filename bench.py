@@ -298,6 +298,10 @@ def run_ours(args, cfg, T, M):
                 dist.barrier()
             torch.cuda.synchronize()
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            # ~100 us of spinning ahead of the start event: the host queues the event and the replays behind it,
+            # so the bracket holds the K steps on the device and not the host's latency to launch the first of
+            # them into an idle GPU (about 8 us per run: 0.04 us per step at K = 200, 1.6 us at K = 5)
+            torch.cuda._sleep(200000)
             e0.record(stream)
             run(steps)
             e1.record(stream)
