@@ -54,6 +54,15 @@ constexpr int kThreads = 192;
 constexpr int kMaxStages = 8;
 constexpr int kSmemLimit = 227 * 1024;      // dynamic shared memory one CTA may opt in to
 constexpr int kNumBMaps = kSegTokens / 16;  // token-tile tensor maps: box heights 16, 32, ..., 128
+// The gate/up pass runs densely over the batch (every selected expert against all tokens, in token tiles of 128,
+// read from the layer input in place) up to 128 tokens, and up to 256 tokens when at most 16 experts are
+// selected: a second token tile re-reads every weight byte from the L2, which costs more than the gathered pass
+// once the weight stream is long (measured at 256 tokens: 72 vs 79 us per layer at budget 16, 102 vs 94 at 32).
+constexpr int kDenseTokens = 2 * kSegTokens;
+constexpr int kDenseTwoTileBudget = 16;
+inline bool dense_batch(int T, int budget, int E) {
+  return T <= kSegTokens || (T <= kDenseTokens && std::min(budget, E) <= kDenseTwoTileBudget);
+}
 constexpr long long kEarlyPollCycles = 400000ll;  // about 200 us: how long a producer looks for the early expert list
 
 // Shared-memory plan for work units of at most kMaxN tokens: the smaller the token tile, the more
@@ -124,6 +133,7 @@ struct FfnParams {
   int T, K, E;
   int I, d;
   int tiles1, tiles2;   // work units per segment: I/64 gate/up tiles, d/128 down tiles
+  int ntt;              // dense gate/up pass: token tiles (of 128 tokens) per (expert, tile); 1 up to 128 tokens
   int steps1, steps2;   // pipeline stages per unit: ceil(d/64 / 2), ceil(kb2 / 2)
   int ksplit;           // down pass: each tile's K range (I) is split over this many units (a power of two, at most kMaxSplit)
   size_t ypair_stride;  // floats between the partial-sum copies of a split down pass
@@ -144,7 +154,13 @@ template <int kSplit, bool kDense>
 __device__ __forceinline__ Unit decode_unit(const FfnParams& p, int u, int u1) {   // u1: gate/up units of the list
   Unit r;
   r.phase = u < u1 ? 1 : 2;
-  const int v = u < u1 ? u : u - u1;
+  int v = u < u1 ? u : u - u1;
+  int tt = 0;   // dense gate/up unit: its token tile; the token tiles of one (expert, tile) are neighbours in the
+                // list, so that they ask for the same weight bytes at about the same time and DRAM sees them once
+  if (kDense && u < u1 && p.ntt > 1) {
+    tt = v % p.ntt;
+    v /= p.ntt;
+  }
   const int tiles = u < u1 ? p.tiles1 : (kSplit > 1 ? p.tiles2 * p.ksplit : p.tiles2);
   const int seg = v / tiles;
   r.seg = seg;
@@ -157,8 +173,8 @@ __device__ __forceinline__ Unit decode_unit(const FfnParams& p, int u, int u1) {
   }
   if (kDense && u < u1) {   // the seg-th expert of the gate/up list, applied to all tokens of the batch in place
     r.expert = p.gu_expert[seg];
-    r.offset = 0;
-    r.count = p.T;
+    r.offset = tt * kSegTokens;
+    r.count = min(kSegTokens, p.T - r.offset);
   } else {
     r.expert = p.seg_expert[seg];
     r.offset = p.seg_offset[seg];
@@ -279,7 +295,7 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
       auto make_final = [&]() {
         pdl_wait();
         const int n_seg = p.counters[kCtrSegments];
-        u1 = (kDense ? p.counters[kCtrGuUnits] : n_seg) * p.tiles1;
+        u1 = (kDense ? p.counters[kCtrGuUnits] * p.ntt : n_seg) * p.tiles1;
         n_units = u1 + n_seg * down_units_per_seg;
         final_known = true;
       };
@@ -292,7 +308,8 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
       int early_units = -1;
       if (kDense) {
         u_cur = blockIdx.x;
-        const int j = u_cur / p.tiles1;
+        const int per_expert = p.tiles1 * p.ntt;   // gate/up units of one expert
+        const int j = u_cur / per_expert;
         int e0 = -1;
         if (j < p.E) {
           const long long t0 = clock64();
@@ -301,7 +318,7 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
             e0 = ld_acquire(p.gu_expert + j);
             if (e0 >= 0) break;
             const int flag = ld_acquire(p.counters + kCtrEarly);
-            if (flag > 0 && u_cur >= (flag - 1) * p.tiles1) break;   // the early list ends before this unit
+            if (flag > 0 && u_cur >= (flag - 1) * per_expert) break;   // the early list ends before this unit
             __nanosleep(128);
             if ((it & 63u) == 63u && clock64() - t0 > kEarlyPollCycles) break;
           }
@@ -310,11 +327,12 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
           un_next.phase = 1;
           un_next.seg = j;
           un_next.expert = e0;
-          un_next.tile = u_cur - j * p.tiles1;
+          const int tt = (u_cur - j * per_expert) % p.ntt;
+          un_next.tile = (u_cur - j * per_expert) / p.ntt;
           un_next.kb0 = 0;
-          un_next.offset = 0;
-          un_next.count = p.T;
-          un_next.npad = (p.T + 15) & ~15;
+          un_next.offset = tt * kSegTokens;
+          un_next.count = min(kSegTokens, p.T - un_next.offset);
+          un_next.npad = (un_next.count + 15) & ~15;
           u1 = n_units = u_cur + 1;   // provisional: the length of the early list is read with the next ticket
         } else {
           make_final();
@@ -345,7 +363,8 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
         // gate/up units wait for the gathered rows; a down unit for the gate/up tiles of its K chunk
         const int32_t* flag = gu ? p.counters + kCtrGather
                                  : p.counters + kCtrReady + ready_index<kSplit, kDense>(p, un, un.kb0);
-        const int need = gu ? n_slots : (kSplit > 1 ? min(p.kb2, p.tiles1 - un.kb0) : p.tiles1);
+        // (a dense gate/up tile is produced once per token tile of the batch)
+        const int need = gu ? n_slots : (kSplit > 1 ? min(p.kb2, p.tiles1 - un.kb0) : p.tiles1) * (kDense ? p.ntt : 1);
         for (int st = 0; st < n_steps; ++st) {
           CYC_T0(t_w);
           if (!mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1u, abort_flag)) {
@@ -418,7 +437,7 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
                 __nanosleep(64);
                 if ((it & 63u) == 63u && clock64() - t0 > kEarlyPollCycles) break;
               }
-              early_units = flag > 0 ? (flag - 1) * p.tiles1 : 0;
+              early_units = flag > 0 ? (flag - 1) * p.tiles1 * p.ntt : 0;
               u1 = n_units = max(early_units, u_cur + 1);
             }
             if (kDense && !final_known && u_next >= n_units) make_final();   // past the early list
@@ -578,8 +597,8 @@ ffn_tc_kernel(const __grid_constant__ MapSet maps1, const __grid_constant__ MapS
         // The loads are in flight while the accumulator is processed.
         int dense_slot = -1;
         if (kDense) {
-          const int t = int(threadIdx.x) - 64;
-          if (t < p.T) {
+          const int t = un.offset + int(threadIdx.x) - 64;   // this thread's token of the unit's token tile
+          if (t < un.offset + un.count) {
 #pragma unroll
             for (int k = 0; k < kMaxK; ++k) {
               if (k < p.K) {
@@ -862,7 +881,7 @@ int choose_split(const base_layer_shape& s, int T, int budget, int ypair_copies)
 }  // namespace
 
 int ffn_tc_static_units(const base_layer_shape& s, int T, int budget, const Workspace& ws) {
-  if (T > 128) return 0;   // batches that gather their tokens take every unit from the ticket counter
+  if (!dense_batch(T, budget, s.E)) return 0;   // batches that gather their tokens take every unit from the ticket counter
   const int segs = max_segments(s.E, T, s.K);
   const int max_units = segs * (s.I / 64 + (s.d / 128) * choose_split(s, T, budget, ws.ypair_copies));
   return std::min(sm_count(), max_units);
@@ -892,7 +911,7 @@ cudaError_t launch_ffn_tc(const base_layer_shape& s, const base_layer_weights& w
   }
   if (!map_rows_kblocks(w.w_down, uint64_t(s.E) * s.d, s.I, 128, kKbPerStage, &m2.a)) return cudaErrorInvalidValue;
   // dense batches (at most 128 tokens, one token tile) read the gate/up token operand from the layer input itself
-  const bool dense = T <= 128;
+  const bool dense = dense_batch(T, budget, s.E);
   const void* x_rows = dense ? hidden : static_cast<const void*>(ws.x_sorted);
   const uint64_t n_x_rows = dense ? uint64_t(T) : slots;
   for (int i = 0; i < kNumBMaps; ++i) {
@@ -926,6 +945,7 @@ cudaError_t launch_ffn_tc(const base_layer_shape& s, const base_layer_weights& w
 #endif
   p.tiles1 = s.I / 64;
   p.tiles2 = s.d / 128;
+  p.ntt = dense ? (T + kSegTokens - 1) / kSegTokens : 1;
   p.steps1 = (s.d / kBlockK + int(kKbPerStage) - 1) / int(kKbPerStage);
   // Few experts with long down rows (d/128 tiles each) leave SMs without a down unit and make every
   // down unit wait for the whole gate/up pass of its segment; the K range (I) is then cut into chunks
@@ -936,7 +956,7 @@ cudaError_t launch_ffn_tc(const base_layer_shape& s, const base_layer_weights& w
   p.kb2 = p.ksplit == 1 ? kb_all
                         : ((kb_all + p.ksplit - 1) / p.ksplit + int(kKbPerStage) - 1) / int(kKbPerStage) * int(kKbPerStage);
   p.steps2 = (p.kb2 + int(kKbPerStage) - 1) / int(kKbPerStage);
-  const int max_units = segs * (p.tiles1 + p.tiles2 * p.ksplit);
+  const int max_units = segs * (p.tiles1 * p.ntt + p.tiles2 * p.ksplit);
   // No expert can receive more tokens than the batch holds, which bounds the token tile.
   cudaError_t e;
   if (T <= 32) e = launch_kernel<32, true>(m1, m2, p, max_units, st);
