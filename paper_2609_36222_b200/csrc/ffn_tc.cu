@@ -55,13 +55,15 @@ constexpr int kMaxStages = 8;
 constexpr int kSmemLimit = 227 * 1024;      // dynamic shared memory one CTA may opt in to
 constexpr int kNumBMaps = kSegTokens / 16;  // token-tile tensor maps: box heights 16, 32, ..., 128
 // The gate/up pass runs densely over the batch (every selected expert against all tokens, in token tiles of 128,
-// read from the layer input in place) up to 128 tokens, and up to 256 tokens when at most 16 experts are
-// selected: a second token tile re-reads every weight byte from the L2, which costs more than the gathered pass
-// once the weight stream is long (measured at 256 tokens: 72 vs 79 us per layer at budget 16, 102 vs 94 at 32).
+// read from the layer input in place) up to 128 tokens, and up to 256 tokens when the selected experts' weights
+// are at most 160 MB: a second token tile re-reads every weight byte from the L2, which costs more than the
+// gathered pass once the weight stream is long (measured at 256 tokens on 9.4 MB experts: 72 vs 79 us per layer
+// at budget 16, 102 vs 94 at budget 32).
 constexpr int kDenseTokens = 2 * kSegTokens;
-constexpr int kDenseTwoTileBudget = 16;
-inline bool dense_batch(int T, int budget, int E) {
-  return T <= kSegTokens || (T <= kDenseTokens && std::min(budget, E) <= kDenseTwoTileBudget);
+constexpr size_t kDenseTwoTileBytes = size_t(160) << 20;   // weight bytes of the selected experts up to which two tiles pay
+inline bool dense_batch(const base_layer_shape& s, int T, int budget) {
+  const size_t stream_bytes = size_t(std::min(budget, s.E)) * 3 * size_t(s.d) * size_t(s.I) * 2;
+  return T <= kSegTokens || (T <= kDenseTokens && stream_bytes <= kDenseTwoTileBytes);
 }
 constexpr long long kEarlyPollCycles = 400000ll;  // about 200 us: how long a producer looks for the early expert list
 
@@ -881,7 +883,7 @@ int choose_split(const base_layer_shape& s, int T, int budget, int ypair_copies)
 }  // namespace
 
 int ffn_tc_static_units(const base_layer_shape& s, int T, int budget, const Workspace& ws) {
-  if (!dense_batch(T, budget, s.E)) return 0;   // batches that gather their tokens take every unit from the ticket counter
+  if (!dense_batch(s, T, budget)) return 0;   // batches that gather their tokens take every unit from the ticket counter
   const int segs = max_segments(s.E, T, s.K);
   const int max_units = segs * (s.I / 64 + (s.d / 128) * choose_split(s, T, budget, ws.ypair_copies));
   return std::min(sm_count(), max_units);
@@ -911,7 +913,7 @@ cudaError_t launch_ffn_tc(const base_layer_shape& s, const base_layer_weights& w
   }
   if (!map_rows_kblocks(w.w_down, uint64_t(s.E) * s.d, s.I, 128, kKbPerStage, &m2.a)) return cudaErrorInvalidValue;
   // dense batches (at most 128 tokens, one token tile) read the gate/up token operand from the layer input itself
-  const bool dense = dense_batch(T, budget, s.E);
+  const bool dense = dense_batch(s, T, budget);
   const void* x_rows = dense ? hidden : static_cast<const void*>(ws.x_sorted);
   const uint64_t n_x_rows = dense ? uint64_t(T) : slots;
   for (int i = 0; i < kNumBMaps; ++i) {
