@@ -212,8 +212,9 @@ int base_moe_decode_layer_noalloc(const base_layer_shape* shape, const base_laye
  * waits for `stream`. Weights stay device-resident. Needs
  * base_moe_decode_layer_host_workspace_bytes(shape, T) bytes of device workspace.
  * h_n_dispatched (host int32, may be NULL) receives the realised active-set size; when it points at the
- * first byte behind h_out's T*d elements inside the same pinned allocation, result and count come back in
- * one copy instead of two.
+ * first byte behind h_out's T*d elements inside the same pinned allocation (memory the driver has mapped for
+ * the device), the kernels write result and count straight into that buffer and no copy back is enqueued;
+ * otherwise they are copied back one after the other.
  */
 size_t base_moe_decode_layer_host_workspace_bytes(const base_layer_shape* shape, int T_max);
 int base_moe_decode_layer_host(const base_layer_shape* shape, const base_layer_weights* weights,

@@ -511,15 +511,20 @@ static int layer_host(const base_layer_shape* shape, const base_layer_weights* w
   c.hidden = d_in;
   c.T = T;
   c.budget = budget;
-  c.out = d_out;
+  // Such a buffer is pinned memory that the driver has mapped for the device (unified addressing): the combine
+  // and the routing kernel then write result and count straight into it, and no copy back is enqueued at all.
+  const bool direct = joined && !(opt && opt->accumulate_out);
+  c.out = direct ? h_out : d_out;
   if (opt) c.opt = *opt;
-  c.dbg.n_dispatched = d_nd;
+  c.dbg.n_dispatched = direct ? h_n_dispatched : d_nd;
   int launches = 0;
   rc = enqueue_layer(c, ws, st, &launches);
   if (rc != BASE_OK) return rc;
   const size_t out_bytes = size_t(T) * shape->d * (c.opt.out_is_fp32 ? 4 : 2);
-  e = cudaMemcpyAsync(h_out, d_out, out_bytes + (joined ? 4 : 0), cudaMemcpyDeviceToHost, st);
-  if (e != cudaSuccess) return cuda_fail(e);
+  if (!direct) {
+    e = cudaMemcpyAsync(h_out, d_out, out_bytes + (joined ? 4 : 0), cudaMemcpyDeviceToHost, st);
+    if (e != cudaSuccess) return cuda_fail(e);
+  }
   if (h_n_dispatched && !joined) {
     e = cudaMemcpyAsync(h_n_dispatched, d_nd, 4, cudaMemcpyDeviceToHost, st);
     if (e != cudaSuccess) return cuda_fail(e);
