@@ -207,6 +207,31 @@ def test_ragged_batch_sizes(T):
     del cfg
 
 
+def test_two_token_tiles_with_the_variants():
+    """129-256 tokens at a small budget: the dense gate/up pass runs in two token tiles per weight tile. Every
+    variant that changes which routes are executed must still land its rows in the right place there."""
+    small = wl.LayerConfig("qwen3_small", d=512, E=128, K=8, I=192, T=200, budgets=(16,))
+    host = HostLayer(small, T=200)
+    dl = device_layer_from_host(host, DEV)
+    check_layer(host, dl, 16, gate_rule=B.GATE_RENORM, fill_rule=B.FILL_DROP)
+    check_layer(host, dl, 12, score_rule=B.SCORE_WEIGHT_SQ)
+    check_layer(host, dl, 16, out_dtype=torch.bfloat16, router_norm=B.ROUTER_NORM_ALL)
+    check_layer(host, dl, 5)                               # fewer experts than K: empty slots
+    # an expert-parallel partition of the same step adds up to the whole
+    hid = bits_to_device(host.hidden_bits, DEV)
+    lg = torch.from_numpy(O.router_logits(host.z, host.router_w, host.router_bias)).to(DEV)
+    whole = torch.empty(200, small.d, dtype=torch.float32, device=DEV)
+    B.base_moe_decode_layer(dl.shape, dl.weights, hid, 16, whole, dl.workspace, router_logits=lg)
+    acc = torch.zeros_like(whole)
+    for first in (0, 64):
+        part = torch.empty_like(whole)
+        B.base_moe_decode_layer(dl.shape, dl.weights, hid, 16, part, dl.workspace, router_logits=lg,
+                                expert_range=(first, 64))
+        acc += part
+    torch.cuda.synchronize()
+    assert (acc - whole).abs().max().item() <= 1e-5 * whole.abs().max().item()
+
+
 @pytest.mark.parametrize("d,E,K,I,T,M", [(256, 32, 8, 128, 1024, 12),      # T and T*K at the compiled limits
                                             (256, 512, 16, 64, 512, 40),      # E, K and T*K at the compiled limits
                                             (256, 512, 16, 64, 3, 512),       # the same expert count, a tiny batch
