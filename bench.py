@@ -37,7 +37,7 @@ sys.path.insert(0, ROOT)
 NOMINAL_HBM_GBS = 8000.0
 # DRAM bytes (read + written) of one FFN launch from the committed ncu capture of the same workload
 # (profiles/ffn_tc_kernel_qwen3_b64_m32.md); other workloads have no capture and report null.
-NCU_FFN_TRAFFIC = {("qwen3", 64, 32): 302.33e6 + 4.21e6}
+NCU_FFN_TRAFFIC = {("qwen3", 64, 32): 302.32e6 + 6.17e6}
 FALLBACK_HBM_GBS = 6650.0
 
 
