@@ -317,6 +317,22 @@ def run_ours(args, cfg, T, M):
         # keep the sampler alive long enough to see the load when the run is very short
         if ms * args.steps < 300 and not args.profile:
             timed(graphs, max(args.steps, int(300 / max(ms, 1e-3))), 0)
+        # spread of the measurement: the chain of one step per replica, replayed 25 times, each replay bracketed by
+        # its own event pair (the pairs cost about 2.6 us per replay, so these sit a little above `value`)
+        per_replay = None
+        if graphs[1] is not None and not args.profile:
+            chain, n_chain = graphs[1], len(graphs[0])
+            pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(25)]
+            with torch.cuda.stream(stream):
+                torch.cuda._sleep(200000)
+                for a, b in pairs:
+                    a.record(stream)
+                    chain.replay()
+                    b.record(stream)
+                stream.synchronize()
+            t = sorted(a.elapsed_time(b) * 1e3 / n_chain for a, b in pairs)
+            per_replay = {"median_us_per_step": t[len(t) // 2], "min_us_per_step": t[0], "max_us_per_step": t[-1],
+                          "replays": len(t), "steps_per_replay": n_chain}
     clk = clocks.summary()
     ms = multi.max_over_ranks(ms, dist, dev)
 
@@ -418,6 +434,8 @@ def run_ours(args, cfg, T, M):
     if ms_dense is not None:
         line["unlimited_budget"] = {"us_per_step": ms_dense * 1e3, "n_dispatched_mean": nd_dense,
                                     "speedup_from_budget": ms_dense / ms}
+    if per_replay is not None:
+        line["per_replay"] = per_replay
     if e2e is not None:
         line["e2e"] = e2e
     if ffn_us is not None:
