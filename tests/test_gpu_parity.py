@@ -471,6 +471,22 @@ def test_stack_shape_batch_and_budget_sweep(T, M):
     torch.cuda.empty_cache()
 
 
+def test_all_48_stack_layers_at_the_headline_point():
+    """Every layer of the 48-layer stack (each has its own seeded weights, router bias and predictor) at batch 64,
+    budget 32, full size, on the oracle's own input for that layer."""
+    cfg = wl.CONFIGS["qwen3_stack"]
+    forced = 0
+    for layer in range(cfg.layers):
+        host = HostLayer(cfg, layer=layer, T=64)
+        dl = device_layer_from_host(host, DEV)
+        rep = check_layer(host, dl, 32)
+        assert rep["n_dispatched"] == 32
+        forced += int(rep["forced"])
+        del dl, host
+        torch.cuda.empty_cache()
+    assert forced <= 4          # near-ties of the 32nd and 33rd score are the exception, not the rule
+
+
 @pytest.mark.parametrize("rule", [B.SCORE_WEIGHT_SQ, B.SCORE_WEIGHT, B.SCORE_STATIC, B.SCORE_TOP1_UNION])
 def test_selection_score_variants(layers, rule):
     """The ablation scores of App. Selection-Rule Ablation behind `score_rule`, same parity bar."""
